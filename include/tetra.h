@@ -1,0 +1,160 @@
+/*
+ * tetra.h -- C ABI of the B200 (sm_100a) Tetra decode-and-multiply library.
+ *
+ * Tetra stores every block of 24 weights as one 48-bit word that names a point
+ * of the Leech lattice (Sec. 3 of the paper); the kernels here expand the word
+ * inside the matrix-vector product (Sec. 5.1) and never materialise weights.
+ *
+ * Conventions for every entry point
+ *   - returns a tetra_status; never throws, never exits the process;
+ *   - "dev" pointers are device memory owned by the caller, "host" pointers are
+ *     host memory owned by the caller; nothing is retained after the call
+ *     returns except where stated;
+ *   - work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = the
+ *     legacy default stream) and the call does not synchronise, except where
+ *     stated;
+ *   - arguments are validated on the host before anything is launched; a
+ *     rejected call launches nothing.
+ *
+ * Word, file order ("canonical"): six little-endian bytes; fields from the
+ * least significant bit: i1[11] i2[11] i3[11] s8[6] b1[1] b2[4] b3[1] p[1] r[1]
+ * g[1] (Sec. 3.3, 3.4; the figure that fixes the positions is not printed, so
+ * this order is this library's).  A matrix in file order is N rows of
+ * nblocks words, tightly packed.
+ */
+#ifndef TETRA_H
+#define TETRA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TETRA_OK = 0,
+    TETRA_ERR_NULL = -1,   /* a required pointer is NULL */
+    TETRA_ERR_SHAPE = -2,  /* N, K, nblocks or count out of range */
+    TETRA_ERR_ALIGN = -3,  /* a pointer is not aligned as documented */
+    TETRA_ERR_BATCH = -4,  /* batch outside [1, TETRA_MAX_BATCH] */
+    TETRA_ERR_CUDA = -5,   /* a CUDA runtime call or launch failed */
+    TETRA_ERR_SIZE = -6,   /* a caller buffer is too small */
+    TETRA_ERR_TABLE = -7   /* the table blob was not written by tetra_build_table */
+} tetra_status;
+
+enum {
+    TETRA_BLOCK = 24,              /* weights per word */
+    TETRA_WORD_BYTES = 6,
+    TETRA_MAX_BATCH = 16,
+    TETRA_PAPER_TABLE_BYTES = 18816 /* 16384 + 2304 + 128, Sec. 3.4 */
+};
+
+/* Human-readable name of a status code (static storage). */
+const char *tetra_status_string(int status);
+
+/* ---- tables (Sec. 3.2-3.4) --------------------------------------------- */
+
+/* Size in bytes of the device table blob tetra_build_table writes: the paper's
+ * 18,816-byte tables followed by the two gains and the derived lookup tables
+ * the kernels stage in shared memory. */
+size_t tetra_table_bytes(void);
+
+/* Builds the decode tables on the host (Golay trellis of Sec. 3.2, rank rows
+ * and middle list of Sec. 3.3, 1/sqrt(16 m) of Sec. 3.4) and copies them to
+ * table_dev (16-byte aligned, at least tetra_table_bytes() bytes).
+ * gain2_host: the two gain values of Eq. (2), or NULL for the defaults
+ * {4.3156, 5.4415}.  Synchronises `stream` before returning. */
+int tetra_build_table(void *table_dev, size_t bytes, const float *gain2_host, void *stream);
+
+/* Writes the paper-format tables (rows u32 | prefixes | branches u16 | suffixes |
+ * 32 floats, all little-endian, TETRA_PAPER_TABLE_BYTES bytes) to host memory.
+ * Host-only; for inspection and checks. */
+int tetra_table_export(void *blob_host, size_t bytes);
+
+/* ---- decode only (Sec. 3.4, Fig. "decode") ----------------------------- */
+
+/* Decodes nblocks words in file order.  codes_dev: 6*nblocks bytes (2-byte
+ * aligned).  y_dev: int8 [nblocks][24] lattice coordinates.  mg_dev (may be
+ * NULL): uint8 [nblocks][2] = shell index m, gain bit g.  Bit-exact integers. */
+int tetra_decode_blocks(const void *codes_dev, const void *table_dev, int8_t *y_dev,
+                        uint8_t *mg_dev, size_t nblocks, void *stream);
+
+/* ---- HBM code layout (Sec. 5.1: the loader only reorders bits and pads) -- */
+
+/* Bytes of the packed device layout of an N x nblocks matrix. */
+size_t tetra_codes_bytes(int N, int nblocks);
+
+/* Reorders file-order words (codes_dev, N*nblocks*6 bytes) into the layout the
+ * GEMV kernels stream (packed_dev, 16-byte aligned, tetra_codes_bytes bytes).
+ * A bijection on each word's 48 bits plus a tiling; no code is expanded.
+ * table_dev: a blob written by tetra_build_table (its trellis map is read). */
+int tetra_pack_codes(const void *codes_dev, const void *table_dev, void *packed_dev, int N,
+                     int nblocks, void *stream);
+
+/* Decodes a packed matrix with the GEMV kernel's own decoder: y_dev int8
+ * [N][nblocks][24], mg_dev (may be NULL) uint8 [N][nblocks][2].  Must equal
+ * tetra_decode_blocks on the file-order words. */
+int tetra_decode_packed(const void *packed_dev, const void *table_dev, int8_t *y_dev,
+                        uint8_t *mg_dev, int N, int nblocks, void *stream);
+
+/* ---- decode-and-multiply (Eq. (2), Sec. 5.1) --------------------------- */
+
+/* y[b][n] = row_scales[n] * sum_blk gain[g]/sqrt(16 m) * sum_j Y[n][blk][j] * x[b][24 blk + j]
+ * with ceil(K/24) words per row and x read as zero beyond K.
+ * codes: packed layout of an N x ceil(K/24) matrix (16-byte aligned).
+ * row_scales: float32 [N].  x: float16 [batch][K] (2-byte aligned; 16-byte
+ * aligned rows are faster).  y: float32 [batch][N], fully overwritten.
+ * Products are exact and accumulation is float32.  1 <= batch <= 16. */
+int tetra_gemv(const void *codes, const float *row_scales, const void *table,
+               const void *x, float *y, int N, int K, int batch, void *stream);
+
+/* The paper's rule for K not a multiple of 24 (Sec. 4.1, 5.1): floor(K/24)
+ * words per row plus an unquantized float16 tail [N][K mod 24], added after the
+ * row-scale multiply.  codes: packed layout of an N x floor(K/24) matrix.
+ * tail may be NULL when K mod 24 == 0. */
+int tetra_gemv_tail(const void *codes, const float *row_scales, const void *table,
+                    const void *x, float *y, int N, int K, int batch,
+                    const void *tail, void *stream);
+
+/* One product of a grouped call. Pointers are device pointers as in tetra_gemv_tail. */
+typedef struct {
+    const void *codes;        /* packed layout, N x floor(K/24) (tail != NULL or K % 24 == 0)
+                                 or N x ceil(K/24) (tail == NULL) */
+    const float *row_scales;  /* [N] */
+    const void *x;            /* float16 [K] */
+    const void *tail;         /* float16 [N][K % 24] or NULL */
+    float *y;                 /* [N] */
+    int32_t N;
+    int32_t K;
+} tetra_problem;
+
+/* Batch-1 products of `count` independent matrices in ONE persistent launch
+ * (one resident set of CTAs walks all of them, the tables staged in shared
+ * memory once).  problems_host: host array, copied before the call returns.
+ * workspace_dev: at least tetra_grouped_workspace_bytes(count) bytes, 16-byte
+ * aligned, owned by the caller and private to this call until it completes. */
+size_t tetra_grouped_workspace_bytes(int count);
+int tetra_gemv_grouped(const tetra_problem *problems_host, int count, const void *table,
+                       void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/* The design the paper describes for its own GPU (Sec. 5.1: a warp per output
+ * row, a lane per block, six table loads per block), kept as a comparison arm
+ * and a cross-check.  codes: file-order words, row_stride bytes per row
+ * (multiple of 2, >= 6*floor(K/24) or 6*ceil(K/24) as in tetra_gemv_tail). */
+int tetra_gemv_paper_design(const void *codes, size_t row_stride, const float *row_scales,
+                            const void *table, const void *x, float *y, int N, int K,
+                            int batch, const void *tail, void *stream);
+
+/* End-to-end convenience: x_host (float16 [batch][K]) is copied to x_stage_dev,
+ * the product runs as tetra_gemv_tail, and y is copied from y_stage_dev to
+ * y_host (float32 [batch][N]), all on `stream`.  Pinned host buffers make the
+ * copies asynchronous.  Does not synchronise. */
+int tetra_gemv_hostio(const void *codes, const float *row_scales, const void *table,
+                      const void *x_host, float *y_host, void *x_stage_dev, float *y_stage_dev,
+                      int N, int K, int batch, const void *tail, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TETRA_H */

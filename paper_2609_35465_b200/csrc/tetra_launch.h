@@ -1,0 +1,37 @@
+// Host-side launch functions shared between the translation units.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace tetra {
+
+// Device-side view of one product; same layout as tetra_problem in tetra.h.
+struct Problem {
+    const void* codes;
+    const float* row_scales;
+    const void* x;
+    const void* tail;
+    float* y;
+    int32_t N;
+    int32_t K;
+};
+static_assert(sizeof(Problem) == 48, "Problem must match tetra_problem");
+
+cudaError_t launch_decode_file(const void* codes, const void* table, int8_t* y, uint8_t* mg, size_t nblocks,
+                               cudaStream_t s);
+cudaError_t launch_pack(const void* codes, const void* table, void* packed, int N, int B, cudaStream_t s);
+cudaError_t launch_decode_packed(const void* packed, const void* table, int8_t* y, uint8_t* mg, int N, int B,
+                                 cudaStream_t s);
+
+// Paper-design GEMV (warp per row, lane per block) on file-order words.
+cudaError_t launch_gemv_paper(const void* codes, size_t row_stride, const float* row_scales, const void* table,
+                              const void* x, float* y, int N, int K, int batch, const void* tail, cudaStream_t s);
+
+// Fast GEMV.  `problems_dev` == nullptr: one product described by `single`
+// (x and y advanced per batch column inside).  Otherwise `count` products read
+// from device memory, batch 1 each.
+cudaError_t launch_gemv_fast(const Problem& single, int batch, const Problem* problems_dev, int count, int max_blocks,
+                             const void* table, cudaStream_t s);
+
+}  // namespace tetra

@@ -1,0 +1,53 @@
+// Host-side construction of the Tetra decode tables (Sec. 3.2-3.4) and of the
+// derived lookup tables the sm_100a kernels stage in shared memory.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+
+namespace tetra {
+
+// The tables exactly as the paper lays them out (Sec. 3.4): 18,816 bytes.
+struct PaperTables {
+    uint32_t rows[4096];      // rank rows, class 0 then class 1, nibble j = rank of coordinate j
+    uint8_t prefixes[128];    // [2*s8 + b1]
+    uint16_t branches[1024];  // [16*s8 + b2] = middle byte | s16 << 8
+    uint8_t suffixes[128];    // [2*s16 + b3]
+    float rsqrt16m[32];       // 1/sqrt(16 m), entry 0 = 0
+};
+static_assert(sizeof(PaperTables) == 18816, "paper table blob is 18,816 bytes");
+
+constexpr uint32_t kTableMagic = 0x54455442u;  // "TETB"
+constexpr uint32_t kTableVersion = 3;
+constexpr int kMiddleClass0 = 1240;            // N0 of Sec. 3.3 (checked at build)
+
+// Everything tetra_build_table copies to the device, in one blob.
+struct DeviceTables {
+    PaperTables paper;          //     0: file-order decode (tetra_decode_blocks, paper-design GEMV)
+    float gain[2];              // 18816
+    uint32_t magic;             // 18824
+    uint32_t version;           // 18828
+    // ---- fast path: everything below is staged in shared memory ------------
+    // Rank rows for PRMT lookup: nibble j = rank (0..3); a coordinate of rank 4
+    // is stored as 8 | 2 (bit 3 flags it for the fix-up path).
+    uint32_t rows_fast[4096];   // 18832
+    uint32_t mid_fast[2048];    // 35216: rows_fast[mix(i2)], indexed by i2 directly
+    // Pattern-byte masks of the Turyn coordinates: bit 4j+2 set where the
+    // Hamming word has coordinate j set; H for a and b, H' for x.
+    uint32_t mask_h[16];        // 43408
+    uint32_t mask_hr[16];       // 43472
+    float scale[2][32];         // 43536: gain[g] / sqrt(16 m)
+    uint32_t pad_[16];          // 43792 (spare)
+    // ---- pack-time only (global memory) ------------------------------------
+    // 12 trellis bits (s8 | b1<<6 | b2<<7 | b3<<11) -> Turyn coordinates a | b<<4 | x<<8.
+    uint16_t trellis_to_abx[4096];
+};
+
+constexpr size_t kFastOffset = offsetof(DeviceTables, rows_fast);
+constexpr size_t kFastBytes = offsetof(DeviceTables, trellis_to_abx) - kFastOffset;
+static_assert(kFastOffset % 16 == 0 && kFastBytes % 16 == 0, "staged part must be 16-byte copyable");
+
+// Fills `out` (gain from gain2, or the defaults when null).  Returns 0, or a
+// negative number naming the structural check that failed (never expected).
+int build_device_tables(DeviceTables* out, const float* gain2);
+
+}  // namespace tetra

@@ -1,0 +1,185 @@
+"""ctypes binding of the Tetra C-ABI library (include/tetra.h).
+
+Argument marshalling only: every step of the decode-and-multiply path runs in
+the CUDA kernels of libtetra_b200.so.  PyTorch supplies device memory and
+streams.  There is no CPU fallback: if the library is missing or a call fails,
+an exception is raised.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtetra_b200.so")
+
+BLOCK = 24
+WORD_BYTES = 6
+MAX_BATCH = 16
+PAPER_TABLE_BYTES = 18816
+
+
+class TetraError(RuntimeError):
+    pass
+
+
+class Problem(C.Structure):
+    """Mirror of tetra_problem."""
+    _fields_ = [("codes", C.c_void_p), ("row_scales", C.c_void_p), ("x", C.c_void_p),
+                ("tail", C.c_void_p), ("y", C.c_void_p), ("N", C.c_int32), ("K", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library; raises if it has not been built (python -m paper_2609_35465_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise TetraError("CUDA library not built: %s is missing (run python -m paper_2609_35465_b200.build)"
+                             % LIB_PATH)
+        L = C.CDLL(LIB_PATH)
+        vp, sz, i32 = C.c_void_p, C.c_size_t, C.c_int
+        L.tetra_status_string.argtypes = [i32]
+        L.tetra_status_string.restype = C.c_char_p
+        L.tetra_table_bytes.argtypes = []
+        L.tetra_table_bytes.restype = sz
+        L.tetra_build_table.argtypes = [vp, sz, vp, vp]
+        L.tetra_table_export.argtypes = [vp, sz]
+        L.tetra_decode_blocks.argtypes = [vp, vp, vp, vp, sz, vp]
+        L.tetra_codes_bytes.argtypes = [i32, i32]
+        L.tetra_codes_bytes.restype = sz
+        L.tetra_pack_codes.argtypes = [vp, vp, vp, i32, i32, vp]
+        L.tetra_decode_packed.argtypes = [vp, vp, vp, vp, i32, i32, vp]
+        L.tetra_gemv.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp]
+        L.tetra_gemv_tail.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp]
+        L.tetra_grouped_workspace_bytes.argtypes = [i32]
+        L.tetra_grouped_workspace_bytes.restype = sz
+        L.tetra_gemv_grouped.argtypes = [vp, i32, vp, vp, sz, vp]
+        L.tetra_gemv_paper_design.argtypes = [vp, sz, vp, vp, vp, vp, i32, i32, i32, vp, vp]
+        L.tetra_gemv_hostio.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise TetraError("%s failed: %s (%d)" % (what, lib().tetra_status_string(rc).decode(), rc))
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(0)
+
+
+# ---------------------------------------------------------------------------
+def tetra_table_bytes() -> int:
+    return lib().tetra_table_bytes()
+
+
+def tetra_table_export() -> bytes:
+    """The paper-format tables (18,816 bytes) as built by the library on the host."""
+    buf = C.create_string_buffer(PAPER_TABLE_BYTES)
+    _check(lib().tetra_table_export(buf, PAPER_TABLE_BYTES), "tetra_table_export")
+    return buf.raw
+
+
+def tetra_build_table(gain=None, device="cuda", stream=None) -> torch.Tensor:
+    """Allocates and fills the device table blob (uint8 tensor)."""
+    table = torch.empty(tetra_table_bytes(), dtype=torch.uint8, device=device)
+    g = None
+    if gain is not None:
+        g = (C.c_float * 2)(float(gain[0]), float(gain[1]))
+    _check(lib().tetra_build_table(_ptr(table), table.numel(), g, _stream(stream)), "tetra_build_table")
+    return table
+
+
+def tetra_decode_blocks(codes: torch.Tensor, table: torch.Tensor, want_mg: bool = True, stream=None):
+    """codes: uint8 [..., 6] file-order words on the device -> (y int8 [n, 24], mg uint8 [n, 2] or None)."""
+    assert codes.dtype == torch.uint8 and codes.is_cuda and codes.is_contiguous()
+    n = codes.numel() // WORD_BYTES
+    y = torch.empty((n, BLOCK), dtype=torch.int8, device=codes.device)
+    mg = torch.empty((n, 2), dtype=torch.uint8, device=codes.device) if want_mg else None
+    _check(lib().tetra_decode_blocks(_ptr(codes), _ptr(table), _ptr(y), _ptr(mg), n, _stream(stream)),
+           "tetra_decode_blocks")
+    return y, mg
+
+
+def tetra_codes_bytes(N: int, nblocks: int) -> int:
+    return lib().tetra_codes_bytes(N, nblocks)
+
+
+def tetra_pack_codes(codes: torch.Tensor, table: torch.Tensor, N: int, nblocks: int, out=None, stream=None):
+    """codes: uint8 [N, nblocks, 6] file order on the device -> packed uint8 tensor."""
+    assert codes.dtype == torch.uint8 and codes.is_cuda and codes.is_contiguous()
+    assert codes.numel() == N * nblocks * WORD_BYTES
+    nbytes = tetra_codes_bytes(N, nblocks)
+    if out is None:
+        out = torch.empty(nbytes, dtype=torch.uint8, device=codes.device)
+    assert out.numel() >= nbytes
+    _check(lib().tetra_pack_codes(_ptr(codes), _ptr(table), _ptr(out), N, nblocks, _stream(stream)),
+           "tetra_pack_codes")
+    return out
+
+
+def tetra_decode_packed(packed: torch.Tensor, table: torch.Tensor, N: int, nblocks: int, want_mg=True, stream=None):
+    y = torch.empty((N, nblocks, BLOCK), dtype=torch.int8, device=packed.device)
+    mg = torch.empty((N, nblocks, 2), dtype=torch.uint8, device=packed.device) if want_mg else None
+    _check(lib().tetra_decode_packed(_ptr(packed), _ptr(table), _ptr(y), _ptr(mg), N, nblocks, _stream(stream)),
+           "tetra_decode_packed")
+    return y, mg
+
+
+def tetra_gemv(codes, row_scales, table, x, y, N: int, K: int, batch: int = 1, stream=None):
+    """Zero-pad rule: ceil(K/24) words per row."""
+    _check(lib().tetra_gemv(_ptr(codes), _ptr(row_scales), _ptr(table), _ptr(x), _ptr(y), N, K, batch,
+                            _stream(stream)), "tetra_gemv")
+    return y
+
+
+def tetra_gemv_tail(codes, row_scales, table, x, y, N: int, K: int, batch: int = 1, tail=None, stream=None):
+    """The paper's rule: floor(K/24) words per row plus a float16 tail."""
+    _check(lib().tetra_gemv_tail(_ptr(codes), _ptr(row_scales), _ptr(table), _ptr(x), _ptr(y), N, K, batch,
+                                 _ptr(tail), _stream(stream)), "tetra_gemv_tail")
+    return y
+
+
+def make_problems(items):
+    """items: iterable of dicts(codes, row_scales, x, tail, y, N, K) of device tensors -> ctypes array."""
+    items = list(items)
+    arr = (Problem * len(items))()
+    for i, it in enumerate(items):
+        arr[i] = Problem(it["codes"].data_ptr(), it["row_scales"].data_ptr(), it["x"].data_ptr(),
+                         it["tail"].data_ptr() if it.get("tail") is not None else None,
+                         it["y"].data_ptr(), it["N"], it["K"])
+    return arr
+
+
+def tetra_grouped_workspace_bytes(count: int) -> int:
+    return lib().tetra_grouped_workspace_bytes(count)
+
+
+def tetra_gemv_grouped(problems, table, workspace: torch.Tensor, stream=None):
+    """problems: ctypes array from make_problems; one persistent launch for all of them."""
+    _check(lib().tetra_gemv_grouped(problems, len(problems), _ptr(table), _ptr(workspace), workspace.numel(),
+                                    _stream(stream)), "tetra_gemv_grouped")
+
+
+def tetra_gemv_paper_design(codes, row_stride: int, row_scales, table, x, y, N: int, K: int, batch: int = 1,
+                            tail=None, stream=None):
+    _check(lib().tetra_gemv_paper_design(_ptr(codes), row_stride, _ptr(row_scales), _ptr(table), _ptr(x), _ptr(y),
+                                         N, K, batch, _ptr(tail), _stream(stream)), "tetra_gemv_paper_design")
+    return y
+
+
+def tetra_gemv_hostio(codes, row_scales, table, x_host, y_host, x_stage, y_stage, N: int, K: int, batch: int = 1,
+                      tail=None, stream=None):
+    """x_host / y_host: pinned CPU tensors; the copies and the product are enqueued on the stream."""
+    _check(lib().tetra_gemv_hostio(_ptr(codes), _ptr(row_scales), _ptr(table), _ptr(x_host), _ptr(y_host),
+                                   _ptr(x_stage), _ptr(y_stage), N, K, batch, _ptr(tail), _stream(stream)),
+           "tetra_gemv_hostio")

@@ -1,0 +1,170 @@
+"""GPU GEMV parity against the FP64 oracle on the same seeded inputs, within
+rel-L2 <= 1e-3 and |delta_n| <= 1e-3 sqrt(sum_k (s_n w_nk x_k)^2) + 1e-6."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_35465_b200 import shapes, synth
+from helpers import assert_gemv_close, make_matrix, oracle_product
+
+pytestmark = pytest.mark.gpu
+GAIN = synth.DEFAULT_GAIN
+
+
+@pytest.fixture(scope="module")
+def tt():
+    from paper_2609_35465_b200 import tetra
+    return tetra
+
+
+@pytest.fixture(scope="module")
+def table(tt):
+    return tt.tetra_build_table(GAIN)
+
+
+def upload(tt, table, m):
+    d = dict(N=m["N"], K=m["K"])
+    codes = torch.from_numpy(m["codes"]).cuda()
+    d["codes_file"] = codes
+    d["codes"] = tt.tetra_pack_codes(codes, table, m["N"], m["B"])
+    d["row_scales"] = torch.from_numpy(m["sigma"]).cuda()
+    d["x"] = torch.from_numpy(m["x"]).cuda()
+    d["tail"] = torch.from_numpy(m["tail"]).cuda() if m["tail"] is not None else None
+    d["y"] = torch.full((m["x"].shape[0], m["N"]), float("nan"), dtype=torch.float32, device="cuda")
+    return d
+
+
+def run_fast(tt, table, m, d):
+    batch = m["x"].shape[0]
+    if m["ntail"]:
+        tt.tetra_gemv_tail(d["codes"], d["row_scales"], table, d["x"], d["y"], m["N"], m["K"], batch, d["tail"])
+    else:
+        tt.tetra_gemv(d["codes"], d["row_scales"], table, d["x"], d["y"], m["N"], m["K"], batch)
+    torch.cuda.synchronize()
+    return d["y"].cpu().numpy()
+
+
+CASES = [
+    # N, K, tail_mode                      (config 0; ragged tails; tiny; wide; zero-pad)
+    (2048, 2304, True),
+    (1024, 2560, True),
+    (1024, 2560, False),
+    (520, 4096, True),
+    (264, 12288, True),
+    (72, 17408, True),
+    (1, 24, True),
+    (7, 48, True),
+    (9, 24 * 33, True),
+    (33, 24 * 31 + 5, True),
+    (33, 24 * 31 + 5, False),
+    (300, 24 * 513, True),
+]
+
+
+@pytest.mark.parametrize("N,K,tail_mode", CASES)
+def test_fast_gemv_matches_oracle(tt, table, orc, N, K, tail_mode):
+    m = make_matrix(31, N * 7 + K, N, K, tail_mode)
+    d = upload(tt, table, m)
+    y = run_fast(tt, table, m, d)
+    assert np.isfinite(y).all()
+    ref = oracle_product(orc, m, GAIN)
+    rel, worst = assert_gemv_close(y[0], ref, "fast %dx%d" % (N, K))
+    # the paper's own check (Sec. 5.1): every row within 1e-5 * sum |w x|
+    assert np.max(np.abs(y[0] - ref["y"]) / ref["abssum"]) < 1e-5
+
+
+@pytest.mark.parametrize("N,K,tail_mode", [(2048, 2304, True), (96, 2560, True), (33, 24 * 31 + 5, False), (5, 24, True)])
+def test_paper_design_gemv_matches_oracle(tt, table, orc, N, K, tail_mode):
+    m = make_matrix(32, N * 7 + K, N, K, tail_mode)
+    d = upload(tt, table, m)
+    tt.tetra_gemv_paper_design(d["codes_file"], 6 * m["B"], d["row_scales"], table, d["x"], d["y"], N, K, 1,
+                               d["tail"])
+    torch.cuda.synchronize()
+    ref = oracle_product(orc, m, GAIN)
+    assert_gemv_close(d["y"].cpu().numpy()[0], ref, "paper design %dx%d" % (N, K))
+
+
+@pytest.mark.parametrize("batch", [2, 5, 16])
+def test_batched_activations(tt, table, orc, batch):
+    m = make_matrix(33, batch, 256, 2560, True, batch=batch)
+    d = upload(tt, table, m)
+    y = run_fast(tt, table, m, d)
+    for b in range(batch):
+        assert_gemv_close(y[b], oracle_product(orc, m, GAIN, batch_index=b), "batch column %d" % b)
+
+
+def test_grouped_launch_one_layer(tt, table, orc):
+    """One Qwen3-4B-shaped layer (config 1) in a single persistent launch, every row checked."""
+    mats = [make_matrix(34, i, mm.N, mm.K, True) for i, mm in enumerate(shapes.QWEN3_4B.layer_matrices())]
+    devs = [upload(tt, table, m) for m in mats]
+    problems = tt.make_problems(devs)
+    ws = torch.empty(tt.tetra_grouped_workspace_bytes(len(devs)), dtype=torch.uint8, device="cuda")
+    tt.tetra_gemv_grouped(problems, table, ws)
+    torch.cuda.synchronize()
+    for m, d in zip(mats, devs):
+        y = d["y"].cpu().numpy()[0]
+        assert_gemv_close(y, oracle_product(orc, m, GAIN), "grouped %dx%d" % (m["N"], m["K"]))
+        # same bits as the single-matrix entry point (the reduction order is fixed)
+        d["y"].fill_(float("nan"))
+        y1 = run_fast(tt, table, m, d)[0]
+        assert np.array_equal(y, y1)
+
+
+def test_special_inputs(tt, table, orc):
+    N, K = 64, 240
+    m = make_matrix(35, 1, N, K, True)
+    m["codes"][:] = 0                                      # origin blocks: y = 0 exactly
+    d = upload(tt, table, m)
+    assert not run_fast(tt, table, m, d).any()
+    m = make_matrix(35, 2, N, K, True)
+    m["x"][:] = 0                                          # zero activations
+    d = upload(tt, table, m)
+    assert not run_fast(tt, table, m, d).any()
+    m = make_matrix(35, 3, N, K, True)                     # unit vectors pick single weights
+    for k in (0, 23, 24, 239):
+        m["x"][:] = 0
+        m["x"][0, k] = 1.0
+        d = upload(tt, table, m)
+        assert_gemv_close(run_fast(tt, table, m, d)[0], oracle_product(orc, m, GAIN), "unit %d" % k)
+    # outlier channels: activations are held exactly down to 2^-12 of their block's largest,
+    # so a block mixing 1000x outliers with ordinary values loses nothing
+    m = make_matrix(35, 4, N, K, True)
+    m["x"][0, 5::24] = (m["x"][0, 5::24].astype(np.float32) * 1000).astype(np.float16)
+    m["x"][0, 30] = np.float16(60000.0)
+    m["x"][0, 31] = np.float16(60000.0 / 4096)
+    d = upload(tt, table, m)
+    y = run_fast(tt, table, m, d)[0]
+    ref = oracle_product(orc, m, GAIN)
+    assert_gemv_close(y, ref, "outlier channels")
+    assert np.max(np.abs(y - ref["y"]) / ref["abssum"]) < 1e-5   # float32 rounding of outlier-sized sums
+    # below that the error is bounded by the step, 2^-23 of the block's largest, per coordinate
+    m = make_matrix(35, 5, N, K, True)
+    m["x"][0, :24:2] = np.float16(6.0e-5)
+    m["x"][0, 5] = np.float16(60000.0)
+    d = upload(tt, table, m)
+    y = run_fast(tt, table, m, d)[0]
+    ref = oracle_product(orc, m, GAIN)
+    Y, mm, g = orc.decode_blocks(m["codes"][:, 0])
+    bound = m["sigma"].astype(np.float64) * GAIN[g] / np.sqrt(16.0 * np.maximum(mm, 1)) * np.abs(Y).sum(axis=1) \
+        * 60000.0 * 2.0 ** -23
+    assert np.all(np.abs(y - ref["y"]) <= bound + 1e-6 * ref["abssum"])
+
+
+def test_reruns_are_bit_identical(tt, table):
+    m = make_matrix(36, 1, 1024, 4096, True)
+    d = upload(tt, table, m)
+    a = run_fast(tt, table, m, d).copy()
+    d["y"].fill_(0)
+    b = run_fast(tt, table, m, d)
+    assert np.array_equal(a, b)
+
+
+def test_hostio_entry_point(tt, table, orc):
+    m = make_matrix(37, 1, 512, 2560, True)
+    d = upload(tt, table, m)
+    xh = torch.from_numpy(m["x"]).pin_memory()
+    yh = torch.empty((1, m["N"]), dtype=torch.float32).pin_memory()
+    xs = torch.empty_like(d["x"])
+    tt.tetra_gemv_hostio(d["codes"], d["row_scales"], table, xh, yh, xs, d["y"], m["N"], m["K"], 1, d["tail"])
+    torch.cuda.synchronize()
+    assert_gemv_close(yh.numpy()[0], oracle_product(orc, m, GAIN), "hostio")
