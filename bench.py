@@ -1,0 +1,326 @@
+#!/usr/bin/env python3
+"""Throughput of the Tetra decode-and-multiply path on B200.
+
+A step is one batch-1 weight pass over every projection matrix of a
+Qwen3-8B-shaped model (252 matrices, about 1.8 GB of 48-bit words, tails,
+scales, activations and results) on synthetic seeded inputs.  The metric is the
+rate at which those algorithmic bytes are consumed (GB/s); the roofline is the
+same bytes over the measured HBM copy bandwidth.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--model qwen3-8b] [--impl ours|reference]
+
+One JSON line on stdout (rank 0).  Under torchrun every rank runs an
+independent replica of the pass on its own GPU (weak scaling, no collective on
+the data path); the time is the maximum over ranks.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "tetra_gemv_batch1_hbm_gbps"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per algorithmic byte of the grouped kernel, from the ncu capture
+# summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on one
+# Qwen3-8B layer, 49 MB of codes; traffic grows in proportion to the matrices read).
+TRAFFIC_PER_ALGORITHMIC_BYTE = None
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML queries)
+# --------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.power = [], set(), []
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "power_w_max": max(self.power) if self.power else None, "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------
+def timed(torch, fn, steps, warmup, stream):
+    """Average milliseconds per call of fn, CUDA events on the launching stream."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def oracle_sample(dp, orc, layers, threads, compare_with=None):
+    """Times the CPU oracle on the first `layers` layers' matrices of the pass.
+    Returns (seconds, bytes processed, worst ratio to the tolerance)."""
+    from tests.helpers import oracle_product  # the tolerance lives with the tests
+    per_layer = 7
+    items = list(range(min(len(dp.items), layers * per_layer)))
+    inputs = [dp.host_inputs(i) for i in items]
+    t0 = time.perf_counter()
+    refs = [oracle_product(orc, m, dp.gain, threads=threads) for m in inputs]
+    dt = time.perf_counter() - t0
+    nbytes = sum(dp.items[i]["bytes"] for i in items)
+    worst = None
+    if compare_with is not None:
+        worst = 0.0
+        for i, ref in zip(items, refs):
+            it = dp.items[i]
+            y = compare_with[it["yoff"]:it["yoff"] + it["N"]].astype(np.float64)
+            bound = 1e-3 * ref["termnorm"] + 1e-6
+            worst = max(worst, float(np.max(np.abs(y - ref["y"]) / bound)))
+    return dt, nbytes, worst, len(items)
+
+
+def run_reference(args, rank, world):
+    """The oracle as it stands, on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2609_35465_b200 import shapes, synth
+    from tests.helpers import make_matrix, oracle_product
+    orc = oracle.get()
+    model = shapes.MODELS[args.model]
+    mats = model.layer_matrices()               # one layer per step: a bounded sample of the pass
+    inputs = [make_matrix(args.seed, i, m.N, m.K, True) for i, m in enumerate(mats)]
+    nbytes = sum(m.N * (m.blocks * 6 + m.ntail * 2 + 8) + m.K * 2 for m in mats)
+    threads = os.cpu_count() or 1
+    for _ in range(args.warmup):
+        [oracle_product(orc, m, synth.DEFAULT_GAIN, threads=threads) for m in inputs]
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        [oracle_product(orc, m, synth.DEFAULT_GAIN, threads=threads) for m in inputs]
+    dt = (time.perf_counter() - t0) / args.steps
+    value = nbytes / dt / 1e9
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s batch-1 weight pass; each step is one layer (7 of %d matrices)"
+                               % (model.name, 7 * model.layers)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": "one layer (7 matrices, %d bytes) per step" % nbytes},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--model", default="qwen3-8b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=0, help="use only the first L layers (profiling runs)")
+    ap.add_argument("--no-extras", action="store_true", help="skip the secondary arms and the CPU baseline")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_35465_b200 import shapes
+    from paper_2609_35465_b200 import build as tbuild
+    from paper_2609_35465_b200.workload import DevicePass
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    if rank == 0:
+        tbuild.build()
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    elif not os.path.exists(tbuild.LIB):
+        tbuild.build()
+
+    model = shapes.MODELS[args.model]
+    mats = model.all_matrices()
+    if args.layers:
+        mats = mats[:7 * args.layers]
+    extras = not args.no_extras and rank == 0
+    dp = DevicePass(mats, seed=args.seed + 1000 * rank, tail_mode=True, keep_file_codes=extras)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- headline: the whole pass as one persistent grouped launch ---------
+    for _ in range(args.warmup):
+        dp.run_grouped()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        dp.run_grouped()
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    y_grouped = dp.y_all.cpu().numpy().copy()
+
+    # ---- end to end: activations from pinned host memory, results back to it
+    e2e_steps = max(3, min(args.steps, 200))
+    e2e_ms = timed(torch, dp.run_grouped_hostio, e2e_steps, 3, stream)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    assert np.array_equal(dp.y_host.numpy(), y_grouped), "host-io result differs from the device-resident run"
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    gbs = dp.algorithmic_bytes / (ms * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": gbs * world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8 products, int32 block sums, f32 accumulation", "data": "synthetic",
+        "config": {"workload": "%s batch-1 weight pass, %d matrices%s" % (
+                       model.name, len(mats), "" if not args.layers else " (first %d layers)" % args.layers),
+                   "launch": "planned list, two launches per pass (tetra_gemv_grouped_run: activation pre-pass + persistent GEMV)",
+                   "k_rule": "floor(K/24) words + float16 tail (the paper's rule)",
+                   "l2": "inputs larger than L2: %.2f GB read per pass" % (dp.algorithmic_bytes / 1e9),
+                   "seed": args.seed},
+        "us_per_pass": ms * 1e3,
+        "weights_per_s": sum(m.N * m.K for m in mats) / (ms * 1e-3) * world,
+        "bits_per_weight_read": dp.algorithmic_bytes * 8 / sum(m.N * m.K for m in mats),
+        "algorithmic_bytes_per_pass": dp.algorithmic_bytes,
+        "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+        "gpu_launches": 2 * args.steps,
+        "clocks": clocks,
+        "e2e": {"value": dp.algorithmic_bytes / (e2e_ms * 1e-3) / 1e9 * world, "unit": UNIT,
+                "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": int(dp.x_host.numel() * 2),
+                "d2h_bytes_per_step": int(dp.y_host.numel() * 4),
+                "api": "tetra_gemv_grouped_hostio: activations from pinned host memory, results to it; "
+                       "codes, scales and tails stay resident in HBM as model weights do"},
+        "roofline": {"bound": "hbm", "kernel": "k_gemv_fast", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                     "frac": gbs / peak, "peak_kind": peak_kind + " copy bandwidth",
+                     "traffic": (None if TRAFFIC_PER_ALGORITHMIC_BYTE is None
+                                 else TRAFFIC_PER_ALGORITHMIC_BYTE * dp.algorithmic_bytes),
+                     "limiter": "ALU pipe (PRMT/LOP3/SHF, 64 lanes/clk/SM), not HBM: see DESIGN.md"},
+        "paper_context": {"L40S_tokens_per_s": [113.8, 95.0, 57.2], "L40S_bits_per_weight": 2.148,
+                          "L40S_kernel_GBps": 278},
+    }
+
+    if extras:
+        # secondary arms, a few repetitions each (not part of `value`)
+        reps = max(3, min(50, args.steps))
+        arms = {}
+        arms["per_matrix_stream_ms"] = timed(torch, dp.run_per_matrix, reps, 3, stream)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=torch.cuda.Stream()):
+            dp.run_per_matrix(stream=torch.cuda.current_stream())
+        arms["per_matrix_graph_ms"] = timed(torch, g.replay, reps, 3, stream)
+        y_single = dp.y_all.cpu().numpy()
+        assert np.linalg.norm(y_single - y_grouped) <= 1e-5 * np.linalg.norm(y_grouped), \
+            "per-matrix launches differ from the planned run"
+        arms["paper_design_stream_ms"] = timed(torch, dp.run_paper_design, max(3, reps // 5), 2, stream)
+        for k in list(arms):
+            arms[k.replace("_ms", "_GBps")] = dp.algorithmic_bytes / (arms[k] * 1e-3) / 1e9
+        out["other_arms"] = arms
+        dp.run_grouped()
+        torch.cuda.synchronize()
+
+        # CPU baseline: the oracle on a bounded sample of the same pass, all host cores
+        import oracle
+        orc = oracle.get()
+        cores = os.cpu_count() or 1
+        dt1, b1, _, _ = oracle_sample(dp, orc, 1, cores)
+        layers = int(max(1, min(model.layers if not args.layers else args.layers, 12.0 / max(dt1, 1e-3))))
+        dt, nb, worst, nmat = oracle_sample(dp, orc, layers, cores, compare_with=y_grouped)
+        out["cpu_baseline"] = {"value": nb / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+                               "sample": "first %d layers (%d matrices, %.3f GB) of the same pass, %.1f s"
+                                         % (layers, nmat, nb / 1e9, dt),
+                               "gpu_vs_oracle_worst_fraction_of_tolerance": worst}
+        if worst is not None and worst > 1.0:
+            raise SystemExit("GPU result outside the tolerance on the CPU-baseline sample: %.3f" % worst)
+
+    print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -129,12 +129,23 @@ typedef struct {
     int32_t K;
 } tetra_problem;
 
-/* Batch-1 products of `count` independent matrices in ONE persistent launch
- * (one resident set of CTAs walks all of them, the tables staged in shared
- * memory once).  problems_host: host array, copied before the call returns.
- * workspace_dev: at least tetra_grouped_workspace_bytes(count) bytes, 16-byte
- * aligned, owned by the caller and private to this call until it completes. */
-size_t tetra_grouped_workspace_bytes(int count);
+/* Batch-1 products of a list of independent matrices from one persistent grid
+ * (the tables staged in shared memory once, every warp walking independent
+ * eight-row units of the whole list).  The list is planned once and run many
+ * times:
+ *   tetra_grouped_workspace_bytes  size of the scratch buffer for this list;
+ *   tetra_gemv_grouped_plan        copies descriptors and index arrays into it
+ *                                  (problems_host is read before the call returns);
+ *   tetra_gemv_grouped_run         one step: a small pre-pass kernel rewrites the
+ *                                  scratch buffer's fixed-point image of every x,
+ *                                  then the persistent kernel computes every y.
+ * workspace_dev: 16-byte aligned device memory owned by the caller; it belongs to
+ * the plan until the last run using it has completed, and runs that share a
+ * workspace must not overlap on the GPU.  tetra_gemv_grouped = plan + run. */
+size_t tetra_grouped_workspace_bytes(const tetra_problem *problems_host, int count);
+int tetra_gemv_grouped_plan(const tetra_problem *problems_host, int count, void *workspace_dev,
+                            size_t workspace_bytes, void *stream);
+int tetra_gemv_grouped_run(void *workspace_dev, const void *table, void *stream);
 int tetra_gemv_grouped(const tetra_problem *problems_host, int count, const void *table,
                        void *workspace_dev, size_t workspace_bytes, void *stream);
 
@@ -153,6 +164,14 @@ int tetra_gemv_paper_design(const void *codes, size_t row_stride, const float *r
 int tetra_gemv_hostio(const void *codes, const float *row_scales, const void *table,
                       const void *x_host, float *y_host, void *x_stage_dev, float *y_stage_dev,
                       int N, int K, int batch, const void *tail, void *stream);
+
+/* A planned run with host activations and results: copies x_bytes from x_host to
+ * x_dev, runs tetra_gemv_grouped_run, copies y_bytes from y_dev to y_host, all on
+ * `stream`.  The planned problems' x and y pointers are expected to point into
+ * [x_dev, x_dev + x_bytes) and [y_dev, y_dev + y_bytes).  Does not synchronise. */
+int tetra_gemv_grouped_hostio(void *workspace_dev, const void *table, const void *x_host,
+                              void *x_dev, size_t x_bytes, float *y_host, const float *y_dev,
+                              size_t y_bytes, void *stream);
 
 #ifdef __cplusplus
 }

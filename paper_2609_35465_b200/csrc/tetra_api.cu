@@ -130,7 +130,7 @@ int tetra_gemv_tail(const void* codes, const float* row_scales, const void* tabl
     const int B = tail_mode ? K / 24 : (K + 23) / 24;
     if (B <= 0 || B > kMaxBlocksPerRow) return TETRA_ERR_SHAPE;
     Problem p{codes, row_scales, x, (K % 24) ? tail : nullptr, y, N, K};
-    return cuda_status(launch_gemv_fast(p, batch, nullptr, 1, B, table, as_stream(stream)));
+    return cuda_status(launch_gemv_fast(p, batch, B, table, as_stream(stream)));
 }
 
 int tetra_gemv(const void* codes, const float* row_scales, const void* table, const void* x, float* y, int N, int K,
@@ -138,31 +138,53 @@ int tetra_gemv(const void* codes, const float* row_scales, const void* table, co
     return tetra_gemv_tail(codes, row_scales, table, x, y, N, K, batch, nullptr, stream);
 }
 
-size_t tetra_grouped_workspace_bytes(int count) { return count > 0 ? size_t(count) * sizeof(Problem) : 0; }
+static int check_problems(const tetra_problem* problems_host, int count) {
+    static_assert(sizeof(tetra_problem) == sizeof(Problem), "descriptor layouts must agree");
+    if (!problems_host) return TETRA_ERR_NULL;
+    if (count <= 0 || count > 65536) return TETRA_ERR_SHAPE;
+    for (int i = 0; i < count; ++i) {
+        const tetra_problem& q = problems_host[i];
+        if (!q.codes || !q.row_scales || !q.x || !q.y) return TETRA_ERR_NULL;
+        if (q.N <= 0 || q.K <= 0) return TETRA_ERR_SHAPE;
+        if (!aligned(q.codes, 16) || !aligned(q.row_scales, 4) || !aligned(q.y, 4) || !aligned(q.x, 2) ||
+            (q.tail && !aligned(q.tail, 2)))
+            return TETRA_ERR_ALIGN;
+        const int B = (q.tail || q.K % 24 == 0) ? q.K / 24 : (q.K + 23) / 24;
+        if (B <= 0 || B > kMaxBlocksPerRow) return TETRA_ERR_SHAPE;
+    }
+    return TETRA_OK;
+}
+
+size_t tetra_grouped_workspace_bytes(const tetra_problem* problems_host, int count) {
+    if (check_problems(problems_host, count) != TETRA_OK) return 0;
+    return grouped_workspace_bytes(reinterpret_cast<const Problem*>(problems_host), count);
+}
+
+int tetra_gemv_grouped_plan(const tetra_problem* problems_host, int count, void* workspace_dev,
+                            size_t workspace_bytes, void* stream) {
+    const int rc = check_problems(problems_host, count);
+    if (rc) return rc;
+    if (!workspace_dev) return TETRA_ERR_NULL;
+    if (!aligned(workspace_dev, 16)) return TETRA_ERR_ALIGN;
+    if (workspace_bytes < grouped_workspace_bytes(reinterpret_cast<const Problem*>(problems_host), count))
+        return TETRA_ERR_SIZE;
+    return cuda_status(grouped_plan(reinterpret_cast<const Problem*>(problems_host), count, workspace_dev,
+                                    workspace_bytes, as_stream(stream)));
+}
+
+int tetra_gemv_grouped_run(void* workspace_dev, const void* table, void* stream) {
+    if (!workspace_dev || !table) return TETRA_ERR_NULL;
+    if (!aligned(workspace_dev, 16) || !aligned(table, 16)) return TETRA_ERR_ALIGN;
+    return cuda_status(grouped_run(workspace_dev, table, as_stream(stream)));
+}
 
 int tetra_gemv_grouped(const tetra_problem* problems_host, int count, const void* table, void* workspace_dev,
                        size_t workspace_bytes, void* stream) {
-    static_assert(sizeof(tetra_problem) == sizeof(Problem), "descriptor layouts must agree");
-    if (!problems_host || !table || !workspace_dev) return TETRA_ERR_NULL;
-    if (count <= 0 || count > 65536) return TETRA_ERR_SHAPE;
-    if (workspace_bytes < tetra_grouped_workspace_bytes(count)) return TETRA_ERR_SIZE;
-    if (!aligned(workspace_dev, 16) || !aligned(table, 16)) return TETRA_ERR_ALIGN;
-    int max_blocks = 0;
-    for (int i = 0; i < count; ++i) {
-        const tetra_problem& q = problems_host[i];
-        const int rc = check_gemv(q.codes, q.row_scales, table, q.x, q.y, q.N, q.K, 1);
-        if (rc) return rc;
-        if (q.tail && !aligned(q.tail, 2)) return TETRA_ERR_ALIGN;
-        const int B = (q.tail || q.K % 24 == 0) ? q.K / 24 : (q.K + 23) / 24;
-        if (B <= 0 || B > kMaxBlocksPerRow) return TETRA_ERR_SHAPE;
-        if (B > max_blocks) max_blocks = B;
-    }
-    cudaError_t e = cudaMemcpyAsync(workspace_dev, problems_host, size_t(count) * sizeof(Problem),
-                                    cudaMemcpyHostToDevice, as_stream(stream));
-    if (e != cudaSuccess) return TETRA_ERR_CUDA;
-    Problem none{};
-    return cuda_status(launch_gemv_fast(none, 1, static_cast<const Problem*>(workspace_dev), count, max_blocks, table,
-                                        as_stream(stream)));
+    if (!table) return TETRA_ERR_NULL;
+    if (!aligned(table, 16)) return TETRA_ERR_ALIGN;
+    const int rc = tetra_gemv_grouped_plan(problems_host, count, workspace_dev, workspace_bytes, stream);
+    if (rc) return rc;
+    return tetra_gemv_grouped_run(workspace_dev, table, stream);
 }
 
 int tetra_gemv_paper_design(const void* codes, size_t row_stride, const float* row_scales, const void* table,
@@ -192,6 +214,18 @@ int tetra_gemv_hostio(const void* codes, const float* row_scales, const void* ta
     if (rc2) return rc2;
     e = cudaMemcpyAsync(y_host, y_stage_dev, size_t(batch) * N * sizeof(float), cudaMemcpyDeviceToHost, s);
     return cuda_status(e);
+}
+
+int tetra_gemv_grouped_hostio(void* workspace_dev, const void* table, const void* x_host, void* x_dev,
+                              size_t x_bytes, float* y_host, const float* y_dev, size_t y_bytes, void* stream) {
+    if (!workspace_dev || !table || !x_host || !x_dev || !y_host || !y_dev) return TETRA_ERR_NULL;
+    if (x_bytes == 0 || y_bytes == 0) return TETRA_ERR_SIZE;
+    if (!aligned(workspace_dev, 16) || !aligned(table, 16)) return TETRA_ERR_ALIGN;
+    cudaStream_t s = as_stream(stream);
+    if (cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return TETRA_ERR_CUDA;
+    const int rc = tetra_gemv_grouped_run(workspace_dev, table, stream);
+    if (rc) return rc;
+    return cuda_status(cudaMemcpyAsync(y_host, y_dev, y_bytes, cudaMemcpyDeviceToHost, s));
 }
 
 }  // extern "C"

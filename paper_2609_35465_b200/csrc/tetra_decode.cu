@@ -94,7 +94,7 @@ __device__ __forceinline__ void emit_block(const FastBlock& fb, int8_t* __restri
                  (uint32_t(y[4 * k + 2] & 0xFF) << 16) | (uint32_t(y[4 * k + 3] & 0xFF) << 24);
     if (mg_out) {
         mg_out[2 * block] = uint8_t(norm >> 4);
-        mg_out[2 * block + 1] = uint8_t(fb.goff >> 7);
+        mg_out[2 * block + 1] = uint8_t((fb.goff >> 7) & 1u);
     }
 }
 
@@ -102,10 +102,9 @@ __global__ void __launch_bounds__(256) k_decode_packed(const uint4* __restrict__
                                                        const DeviceTables* __restrict__ tab,
                                                        int8_t* __restrict__ y_out, uint8_t* __restrict__ mg_out,
                                                        int N, int B) {
-    extern __shared__ uint4 sm_tab4[];
-    stage_fast_tables(tab, sm_tab4);
+    extern __shared__ __align__(16) unsigned char smem[];
+    const uint32_t sm_tab = smem_u32(stage_fast_tables(tab, smem));
     __syncthreads();
-    const uint32_t sm_tab = smem_u32(sm_tab4);
     const int groups = (N + 7) / 8;
     const size_t total = size_t(groups) * B;
     for (size_t t = blockIdx.x * size_t(blockDim.x) + threadIdx.x; t < total;
@@ -155,7 +154,7 @@ cudaError_t launch_pack(const void* codes, const void* table, void* packed, int 
 cudaError_t launch_decode_packed(const void* packed, const void* table, int8_t* y, uint8_t* mg, int N, int B,
                                  cudaStream_t s) {
     const size_t items = size_t((N + 7) / 8) * B;
-    k_decode_packed<<<grid_for(items, 256, 148 * 8), 256, kFastBytes, s>>>(
+    k_decode_packed<<<grid_for(items, 256, 148 * 4), 256, kTableSmemBytes, s>>>(
         static_cast<const uint4*>(packed), static_cast<const DeviceTables*>(table), y, mg, N, B);
     return cudaGetLastError();
 }

@@ -36,14 +36,16 @@ __device__ __forceinline__ int dp4a_su(uint32_t a, uint32_t b, int c) {  // sign
     asm("dp4a.s32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
 }
+// Loads from the staged tables: they never change after staging, so the loads
+// are not volatile and the compiler may schedule them freely.
 __device__ __forceinline__ uint32_t lds32(uint32_t saddr) {
     uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(saddr));
+    asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(saddr));
     return v;
 }
 __device__ __forceinline__ float lds32f(uint32_t saddr) {
     float v;
-    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(saddr));
+    asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(saddr));
     return v;
 }
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -117,17 +119,28 @@ __device__ __forceinline__ void file_to_device_word(uint64_t w, const uint16_t* 
 
 // Byte offsets of the staged tables inside the shared-memory copy of the fast part.
 constexpr uint32_t kSmRows = 0;
-constexpr uint32_t kSmMid = kSmRows + 4096 * 4;
-constexpr uint32_t kSmMaskH = kSmMid + 2048 * 4;
-constexpr uint32_t kSmMaskHr = kSmMaskH + 64;
-constexpr uint32_t kSmScale = kSmMaskHr + 64;
+constexpr uint32_t kSmMid = 16384;
+constexpr uint32_t kSmScale = 24576;
+constexpr uint32_t kSmMaskH = 24832;
+constexpr uint32_t kSmMaskHr = 24896;
+constexpr uint32_t kSmAlign = 16384;  // the staged copy starts on a 16 KiB boundary of shared memory
+static_assert(kSmMid == offsetof(DeviceTables, mid_fast) - kFastOffset, "staged layout");
 static_assert(kSmScale == offsetof(DeviceTables, scale) - kFastOffset, "staged layout");
+static_assert(kSmMaskH == offsetof(DeviceTables, mask_h) - kFastOffset, "staged layout");
+static_assert(kSmMaskHr == offsetof(DeviceTables, mask_hr) - kFastOffset, "staged layout");
 
-// Copies the staged part of the tables into shared memory (all threads of the CTA).
-__device__ __forceinline__ void stage_fast_tables(const DeviceTables* tab, uint4* sm) {
+// Copies the staged part of the tables to the first 16 KiB boundary of the
+// CTA's dynamic shared memory (all threads; the caller synchronises) and returns
+// that address.  The launch must reserve kFastBytes + kSmAlign bytes for it.
+__device__ __forceinline__ unsigned char* stage_fast_tables(const DeviceTables* tab, unsigned char* smem) {
+    const uint32_t s = smem_u32(smem);
+    unsigned char* base = smem + (((s + kSmAlign - 1) & ~(kSmAlign - 1)) - s);
     const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(tab) + kFastOffset);
-    for (uint32_t i = threadIdx.x; i < kFastBytes / 16; i += blockDim.x) sm[i] = src[i];
+    uint4* dst = reinterpret_cast<uint4*>(base);
+    for (uint32_t i = threadIdx.x; i < kFastBytes / 16; i += blockDim.x) dst[i] = src[i];
+    return base;
 }
+constexpr uint32_t kTableSmemBytes = uint32_t(kFastBytes) + kSmAlign;
 
 // PRMT pool of the p = 0 image, indexed by rank | c << 2:
 //   c = 0: 0, 4, -4, 8     c = 1: 2, -2, 6, -6
@@ -142,34 +155,38 @@ struct FastBlock {
     uint32_t sel1;    // PRMT selectors (rank | c << 2 per nibble), for the fix-up
     uint32_t sel3;
     uint32_t p13;     // p << 13
-    uint32_t goff;    // g * 128: byte offset of the gain's half of the scale table
+    uint32_t goff;    // shared-memory address of the gain's half of the scale table (bit 7 = g)
 };
 
 // HI = false: w1 sits in bits 0..15 of `w1pair`; HI = true: in bits 16..31.
+// sm_tab: shared-memory address of the staged tables, a multiple of 16 KiB, so
+// that every index is merged with its table's address by the same LOP3 that
+// masks it.
 template <bool HI>
 __device__ __forceinline__ void fast_decode(uint32_t sm_tab, uint32_t w0, uint32_t w1pair, FastBlock& out) {
-    const uint32_t addr1 = (w0 << 2) & 0x3FFCu;          // (i1 | r << 11) * 4
-    const uint32_t addr3p = (w0 >> 10) & 0x3FFCu;        // (i3 | q << 11) * 4
-    const uint32_t a4 = (w0 >> 22) & 0x3Cu;
-    const uint32_t b4 = (w0 >> 26) & 0x3Cu;
+    const uint32_t addr1 = ((w0 << 2) & 0x3FFCu) | (sm_tab + kSmRows);    // (i1 | r << 11) * 4
+    const uint32_t addr3p = ((w0 >> 10) & 0x3FFCu) | (sm_tab + kSmRows);  // (i3 | q << 11) * 4
+    const uint32_t a4 = ((w0 >> 22) & 0x3Cu) | (sm_tab + kSmMaskH);
+    const uint32_t b4 = ((w0 >> 26) & 0x3Cu) | (sm_tab + kSmMaskH);
     uint32_t addr2, x4;
     if (HI) {
-        addr2 = (w1pair >> 14) & 0x1FFCu;
-        x4 = (w1pair >> 25) & 0x3Cu;
-        out.goff = (w1pair >> 24) & 0x80u;
+        addr2 = ((w1pair >> 14) & 0x1FFCu) | (sm_tab + kSmMid);
+        x4 = ((w1pair >> 25) & 0x3Cu) | (sm_tab + kSmMaskHr);
+        out.goff = ((w1pair >> 24) & 0x80u) | (sm_tab + kSmScale);
     } else {
-        addr2 = (w1pair << 2) & 0x1FFCu;
-        x4 = (w1pair >> 9) & 0x3Cu;
-        out.goff = (w1pair >> 8) & 0x80u;
+        addr2 = ((w1pair << 2) & 0x1FFCu) | (sm_tab + kSmMid);
+        x4 = ((w1pair >> 9) & 0x3Cu) | (sm_tab + kSmMaskHr);
+        out.goff = ((w1pair >> 8) & 0x80u) | (sm_tab + kSmScale);
     }
-    const uint32_t row1 = lds32(sm_tab + kSmRows + addr1);
-    const uint32_t row2 = lds32(sm_tab + kSmMid + addr2);
-    // delta = [i2 >= 1240]: bit 11 of i2 + 808, i.e. bit 13 of the byte offset; Eq. (3)
+    const uint32_t row1 = lds32(addr1);
+    const uint32_t row2 = lds32(addr2);
+    // delta = [i2 >= 1240]: bit 11 of i2 + 808, i.e. bit 13 of the byte offset; Eq. (3).
+    // (the table bases are multiples of 8 KiB, so they do not disturb bits 0..12 of the sum)
     const uint32_t addr3 = addr3p ^ ((addr2 + 808u * 4u) & 0x2000u);
-    const uint32_t row3 = lds32(sm_tab + kSmRows + addr3);
-    const uint32_t ma = lds32(sm_tab + kSmMaskH + a4);
-    const uint32_t mb = lds32(sm_tab + kSmMaskH + b4);
-    const uint32_t mx = lds32(sm_tab + kSmMaskHr + x4);
+    const uint32_t row3 = lds32(addr3);
+    const uint32_t ma = lds32(a4);
+    const uint32_t mb = lds32(b4);
+    const uint32_t mx = lds32(x4);
     const uint32_t sel1 = row1 ^ ma ^ mx;
     const uint32_t sel2 = row2 ^ mb ^ mx;
     const uint32_t sel3 = row3 ^ (ma ^ mb) ^ mx;

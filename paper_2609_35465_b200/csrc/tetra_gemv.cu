@@ -4,7 +4,8 @@
 //                 per output row, a lane per block, the six table loads of
 //                 Fig. "decode", FP32 multiply-accumulate, shuffle reduction.
 //                 Kept as a comparison arm and cross-check.
-//   k_gemv_fast   the B200 design: a lane owns one block column and keeps its
+//   k_gemv_fast / k_gemv_units
+//                 the B200 design: a lane owns one block column and keeps its
 //                 24 activations in registers as 24-bit fixed point (three int8
 //                 planes, power-of-two step per block column, so float16 inputs
 //                 within 2^12 of the column's largest are held exactly); it
@@ -13,8 +14,18 @@
 //                 a block are exact integers, one rounding when the block's sum
 //                 becomes a float, FP32 accumulation across blocks.  The ALU
 //                 pipe only unpacks fields; the integer-MAD pipe does the
-//                 arithmetic.  One persistent grid serves one matrix or a list.
+//                 arithmetic.
+//                 k_gemv_fast serves one matrix per launch and needs no
+//                 scratch memory (every CTA quantises x for itself).
+//                 k_gemv_units serves a planned list of matrices from one
+//                 persistent grid: k_prepare_x first writes the fixed-point
+//                 activations of every matrix to the plan's scratch area, then
+//                 every warp walks independent units (eight rows of one matrix,
+//                 all columns), so no warp ever waits for another.
 #include <cuda_fp16.h>
+
+#include <cstdlib>
+#include <cstring>
 
 #include "tetra_device.cuh"
 #include "tetra_launch.h"
@@ -86,72 +97,66 @@ cudaError_t launch_gemv_paper(const void* codes, size_t row_stride, const float*
 }
 
 // ===========================================================================
-// Fast kernel
+// Fast kernels: shared pieces
 // ===========================================================================
 constexpr int kFastThreads = 512;
 constexpr int kFastWarps = kFastThreads / 32;
 constexpr int kRedStride = 36;                 // floats per row of the transpose buffer (32 + pad)
-constexpr int kRowAccFloats = 2048;            // per-CTA buffer of per-(column group, row) sums
+constexpr int kRedFloats = 8 * kRedStride;     // per warp
+constexpr int kRowAccFloats = 2048;            // k_gemv_fast: per-CTA buffer of per-(column group, row) sums
 constexpr int kXqBytesPerCol = 80;             // 3 planes x 24 bytes, step, sum
-constexpr uint32_t kXqHi = 0, kXqMid = 24, kXqLo = 48, kXqStep = 72, kXqSum = 76;
+constexpr uint32_t kXqHi = 0, kXqMid = 24, kXqLo = 48;
 
-struct FastSmemLayout {
-    uint32_t tab, xq, red, rowacc, total;
-};
-__host__ __device__ inline FastSmemLayout fast_smem_layout(int max_blocks) {
-    FastSmemLayout L;
-    L.tab = 0;
-    L.xq = uint32_t(kFastBytes);
-    L.red = L.xq + uint32_t(max_blocks) * kXqBytesPerCol;
-    L.rowacc = L.red + kFastWarps * 8 * kRedStride * 4;
-    L.total = L.rowacc + kRowAccFloats * 4;
-    return L;
-}
-
-// Fixed-point image of this matrix's activations in shared memory.  Per block
-// column: step = 2^(E-22) with 2^E <= max|x| < 2^(E+1); q_j = rint(x_j / step),
-// |q_j| < 2^23, stored as three byte planes (bits 23..16 signed, 15..8 and 7..0
-// unsigned), four coordinates per 32-bit word; then the step and sum(q_j).
-// A float16 x_j is held exactly when |x_j| >= 2^(E-12); smaller ones are
-// rounded to a multiple of the step.  Every CTA does this for itself.
-__device__ __forceinline__ void quantise_x(const __half* __restrict__ x, int K, int B, unsigned char* smem,
-                                           const FastSmemLayout& L) {
-    for (int c = threadIdx.x; c < B; c += blockDim.x) {
-        float v[24];
-        float mx = 0.f;
+// Fixed-point image of one block column of activations (20 words).
+// step = 2^(E-22) with 2^E <= max|x| < 2^(E+1); q_j = rint(x_j / step), |q_j| < 2^23,
+// stored as three byte planes (bits 23..16 signed, 15..8 and 7..0 unsigned), four
+// coordinates per 32-bit word: words 0..5 high, 6..11 middle, 12..17 low plane;
+// word 18 = step (float), word 19 = sum(q_j).  A float16 x_j is held exactly when
+// |x_j| >= 2^(E-12); smaller ones are rounded to a multiple of the step.
+__device__ __forceinline__ void quantise_column(const __half* __restrict__ x, int K, int c, uint32_t out[20]) {
+    float v[24];
+    const int k0 = 24 * c;
+    if (k0 + 24 <= K && ((reinterpret_cast<uintptr_t>(x) & 15) == 0)) {  // 48-byte column, 16-byte aligned
+        const uint4* src = reinterpret_cast<const uint4*>(x + k0);
 #pragma unroll
-        for (int j = 0; j < 24; ++j) {
-            const int k = 24 * c + j;
-            v[j] = k < K ? __half2float(x[k]) : 0.f;
-            mx = fmaxf(mx, fabsf(v[j]));
-        }
-        const uint32_t e = __float_as_uint(mx) >> 23;  // biased exponent of the largest (finite float16 input)
-        const float step = mx > 0.f ? __uint_as_float((e - 22u) << 23) : 0.f;
-        const float inv = mx > 0.f ? __uint_as_float((276u - e) << 23) : 0.f;
-        int sum = 0;
-        uint32_t hi[6], mid[6], lo[6];
+        for (int i = 0; i < 3; ++i) {
+            const uint4 u = __ldg(src + i);
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
-        for (int k = 0; k < 6; ++k) {
-            hi[k] = mid[k] = lo[k] = 0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int q = __float2int_rn(v[4 * k + i] * inv);
-                sum += q;
-                hi[k] |= (uint32_t(q >> 16) & 0xFFu) << (8 * i);
-                mid[k] |= (uint32_t(q >> 8) & 0xFFu) << (8 * i);
-                lo[k] |= (uint32_t(q) & 0xFFu) << (8 * i);
+            for (int j = 0; j < 4; ++j) {
+                const __half2 h = *reinterpret_cast<const __half2*>(&w[j]);
+                v[8 * i + 2 * j] = __low2float(h);
+                v[8 * i + 2 * j + 1] = __high2float(h);
             }
         }
-        uint32_t* dst = reinterpret_cast<uint32_t*>(smem + L.xq + c * kXqBytesPerCol);
+    } else {
 #pragma unroll
-        for (int k = 0; k < 6; ++k) {
-            dst[k] = hi[k];
-            dst[6 + k] = mid[k];
-            dst[12 + k] = lo[k];
-        }
-        reinterpret_cast<float*>(dst)[18] = step;
-        reinterpret_cast<int*>(dst)[19] = sum;
+        for (int j = 0; j < 24; ++j) v[j] = k0 + j < K ? __half2float(x[k0 + j]) : 0.f;
     }
+    float mx = 0.f;
+#pragma unroll
+    for (int j = 0; j < 24; ++j) mx = fmaxf(mx, fabsf(v[j]));
+    const uint32_t e = __float_as_uint(mx) >> 23;  // biased exponent of the largest (finite float16 input)
+    const float step = mx > 0.f ? __uint_as_float((e - 22u) << 23) : 0.f;
+    const float inv = mx > 0.f ? __uint_as_float((276u - e) << 23) : 0.f;
+    int sum = 0;
+#pragma unroll
+    for (int k = 0; k < 6; ++k) {
+        uint32_t hi = 0, mid = 0, lo = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int q = __float2int_rn(v[4 * k + i] * inv);
+            sum += q;
+            hi |= (uint32_t(q >> 16) & 0xFFu) << (8 * i);
+            mid |= (uint32_t(q >> 8) & 0xFFu) << (8 * i);
+            lo |= (uint32_t(q) & 0xFFu) << (8 * i);
+        }
+        out[k] = hi;
+        out[6 + k] = mid;
+        out[12 + k] = lo;
+    }
+    out[18] = __float_as_uint(step);
+    out[19] = uint32_t(sum);
 }
 
 struct LaneX {
@@ -162,21 +167,29 @@ struct LaneX {
     int sum;          // sum of q over the 24 coordinates
 };
 
-// q of one coordinate, read back from the planes in shared memory (fix-up path only).
-__device__ __forceinline__ int xq_coord(uint32_t xq_col, int coord) {
-    int h;
-    uint32_t m, l;
-    asm volatile("ld.shared.s8 %0, [%1];" : "=r"(h) : "r"(xq_col + kXqHi + uint32_t(coord)));
-    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(m) : "r"(xq_col + kXqMid + uint32_t(coord)));
-    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(l) : "r"(xq_col + kXqLo + uint32_t(coord)));
-    return h * 65536 + int(m << 8 | l);
+__device__ __forceinline__ void lane_x_from_words(const uint32_t q[20], bool active, LaneX& X) {
+#pragma unroll
+    for (int k = 0; k < 6; ++k) {
+        X.hi[k] = active ? q[k] : 0u;
+        X.mid[k] = active ? q[6 + k] : 0u;
+        X.lo[k] = active ? q[12 + k] : 0u;
+    }
+    X.step = active ? __uint_as_float(q[18]) : 0.f;
+    X.sum = active ? int(q[19]) : 0;
+}
+
+// q of one coordinate, read back from a column's record (fix-up path only; the
+// record may sit in shared or in global memory).
+__device__ __forceinline__ int xq_coord(const unsigned char* rec, int coord) {
+    const int h = reinterpret_cast<const signed char*>(rec)[kXqHi + coord];
+    return h * 65536 + (int(rec[kXqMid + coord]) << 8 | int(rec[kXqLo + coord]));
 }
 
 // One block: device word -> contribution scale_b * sum_j y_j x_j (Eq. (2) without
-// the row scale).  xq_col: shared-memory address of this column's fixed-point image.
+// the row scale).  xq_rec: this column's fixed-point record.
 template <bool HI>
 __device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint32_t w1pair, const LaneX& X,
-                                             uint32_t xq_col) {
+                                             const unsigned char* xq_rec) {
     FastBlock fb;
     fast_decode<HI>(sm_tab, w0, w1pair, fb);
     int dh = 0, dm = 0, dl = 0, n2 = 0, n1 = 0;
@@ -194,14 +207,14 @@ __device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint3
         if (fb.flags1) {
             int j, dy, dsq;
             rank4_fix(fb.flags1, fb.sel1, &j, &dy, &dsq);
-            dot += dy * xq_coord(xq_col, j);
+            dot += dy * xq_coord(xq_rec, j);
             n2 += dsq;
             n1 += dy;
         }
         if (fb.flags3) {
             int j, dy, dsq;
             rank4_fix(fb.flags3, fb.sel3, &j, &dy, &dsq);
-            dot += dy * xq_coord(xq_col, 16 + j);
+            dot += dy * xq_coord(xq_rec, 16 + j);
             n2 += dsq;
             n1 += dy;
         }
@@ -210,37 +223,80 @@ __device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint3
         dot = X.sum - dot;
         n2 = n2 - 2 * n1 + 24;
     }
-    // n2 = 16 m; the scale table holds gain[g] / sqrt(16 m) at byte 128 g + 4 m
-    const float scale = lds32f(sm_tab + kSmScale + fb.goff + (uint32_t(n2) >> 2));
+    // n2 = 16 m; the scale table holds gain[g] / sqrt(16 m) at 128 g + 4 m
+    const float scale = lds32f(fb.goff + (uint32_t(n2) >> 2));
     return float(dot) * (scale * X.step);
 }
 
+// The eight blocks of one 48-byte record (rows 8G..8G+7 of one column).
+__device__ __forceinline__ void record_values(uint32_t sm_tab, const uint4& a, const uint4& b, const uint4& h,
+                                              const LaneX& X, const unsigned char* xq_rec, float v[8]) {
+    v[0] = block_value<false>(sm_tab, a.x, h.x, X, xq_rec);
+    v[1] = block_value<true>(sm_tab, a.y, h.x, X, xq_rec);
+    v[2] = block_value<false>(sm_tab, a.z, h.y, X, xq_rec);
+    v[3] = block_value<true>(sm_tab, a.w, h.y, X, xq_rec);
+    v[4] = block_value<false>(sm_tab, b.x, h.z, X, xq_rec);
+    v[5] = block_value<true>(sm_tab, b.y, h.z, X, xq_rec);
+    v[6] = block_value<false>(sm_tab, b.z, h.w, X, xq_rec);
+    v[7] = block_value<true>(sm_tab, b.w, h.w, X, xq_rec);
+}
+
+// Sums v[r] over the 32 lanes for r = 0..7 through the warp's shared-memory
+// buffer.  Afterwards lane l holds, for row l / 4, the partial sum over lanes
+// 8 (l % 4) .. 8 (l % 4) + 7; the caller finishes with two shuffles.
+__device__ __forceinline__ float transpose_partial(float* red, int lane, const float v[8]) {
+    __syncwarp();
+#pragma unroll
+    for (int r = 0; r < 8; ++r) red[r * kRedStride + lane] = v[r];
+    __syncwarp();
+    const float4 s0 = *reinterpret_cast<const float4*>(red + (lane >> 2) * kRedStride + 8 * (lane & 3));
+    const float4 s1 = *reinterpret_cast<const float4*>(red + (lane >> 2) * kRedStride + 8 * (lane & 3) + 4);
+    return ((s0.x + s0.y) + (s0.z + s0.w)) + ((s1.x + s1.y) + (s1.z + s1.w));
+}
+
+// ===========================================================================
+// k_gemv_fast: one matrix per launch, no scratch memory
+// ===========================================================================
+struct FastSmemLayout {
+    uint32_t xq, red, rowacc, total;  // offsets from the 16 KiB-aligned table copy
+};
+__host__ __device__ inline FastSmemLayout fast_smem_layout(int max_blocks) {
+    FastSmemLayout L;
+    L.xq = uint32_t(kFastBytes);
+    L.red = L.xq + uint32_t(max_blocks) * kXqBytesPerCol;
+    L.rowacc = L.red + kFastWarps * kRedFloats * 4;
+    L.total = L.rowacc + kRowAccFloats * 4 + kSmAlign;
+    return L;
+}
+
 __global__ void __launch_bounds__(kFastThreads, 1)
-k_gemv_fast(const DeviceTables* __restrict__ tab, const Problem* __restrict__ problems, const Problem single,
-            int count, int batch, int max_blocks) {
-    extern __shared__ __align__(16) unsigned char smem[];
+k_gemv_fast(const DeviceTables* __restrict__ tab, const Problem single, int batch, int max_blocks) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
     const FastSmemLayout L = fast_smem_layout(max_blocks);
-    stage_fast_tables(tab, reinterpret_cast<uint4*>(smem));
+    unsigned char* smem = stage_fast_tables(tab, smem_raw);
     const uint32_t sm_tab = smem_u32(smem);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float* red = reinterpret_cast<float*>(smem + L.red) + warp * 8 * kRedStride;
+    float* red = reinterpret_cast<float*>(smem + L.red) + warp * kRedFloats;
     float* rowacc = reinterpret_cast<float*>(smem + L.rowacc);
 
-    const int njobs = problems ? count : batch;
-    for (int job = 0; job < njobs; ++job) {
-        Problem P = problems ? problems[job] : single;
-        if (!problems) {  // batch column `job` of the single product
-            P.x = static_cast<const __half*>(P.x) + size_t(job) * P.K;
-            P.y = P.y + size_t(job) * P.N;
-        }
+    for (int job = 0; job < batch; ++job) {  // batch column `job`
+        Problem P = single;
+        P.x = static_cast<const __half*>(P.x) + size_t(job) * P.K;
+        P.y = P.y + size_t(job) * P.N;
         const int ntail = P.tail ? P.K % 24 : 0;
         const int B = P.tail ? P.K / 24 : (P.K + 23) / 24;
         const int groups = (P.N + 7) / 8;
         const int g_begin = int((long long)blockIdx.x * groups / gridDim.x);
         const int g_end = int((long long)(blockIdx.x + 1) * groups / gridDim.x);
         const int CG = (B + 31) / 32;
-        __syncthreads();  // previous job's epilogue is done with xq / rowacc; tables are staged
-        if (g_begin < g_end) quantise_x(static_cast<const __half*>(P.x), P.K, B, smem, L);
+        __syncthreads();  // previous column's epilogue is done with xq / rowacc; tables are staged
+        for (int c = threadIdx.x; c < B; c += blockDim.x) {
+            uint32_t q[20];
+            quantise_column(static_cast<const __half*>(P.x), P.K, c, q);
+            uint4* dst = reinterpret_cast<uint4*>(smem + L.xq + c * kXqBytesPerCol);
+#pragma unroll
+            for (int k = 0; k < 5; ++k) dst[k] = make_uint4(q[4 * k], q[4 * k + 1], q[4 * k + 2], q[4 * k + 3]);
+        }
         __syncthreads();
 
         const bool narrow = CG <= kFastWarps;
@@ -258,23 +314,17 @@ k_gemv_fast(const DeviceTables* __restrict__ tab, const Problem* __restrict__ pr
                 for (int cg = narrow ? warp % CG : warp; cg < CG; cg += cg_step) {
                     const int col = cg * 32 + lane;
                     const bool active = col < B;
-                    const uint32_t xq_col = sm_tab + L.xq + uint32_t(active ? col : 0) * kXqBytesPerCol;
+                    const unsigned char* xq_rec = smem + L.xq + (active ? col : 0) * kXqBytesPerCol;
                     LaneX X;
                     {
                         uint32_t q[20];
+                        const uint4* src = reinterpret_cast<const uint4*>(xq_rec);
 #pragma unroll
-                        for (int k = 0; k < 5; ++k)
-                            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                                         : "=r"(q[4 * k]), "=r"(q[4 * k + 1]), "=r"(q[4 * k + 2]), "=r"(q[4 * k + 3])
-                                         : "r"(xq_col + 16u * k));
-#pragma unroll
-                        for (int k = 0; k < 6; ++k) {
-                            X.hi[k] = active ? q[k] : 0u;
-                            X.mid[k] = active ? q[6 + k] : 0u;
-                            X.lo[k] = active ? q[12 + k] : 0u;
+                        for (int k = 0; k < 5; ++k) {
+                            const uint4 u = src[k];
+                            q[4 * k] = u.x; q[4 * k + 1] = u.y; q[4 * k + 2] = u.z; q[4 * k + 3] = u.w;
                         }
-                        X.step = active ? __uint_as_float(q[18]) : 0.f;
-                        X.sum = active ? int(q[19]) : 0;
+                        lane_x_from_words(q, active, X);
                     }
                     const uint4 zero4 = make_uint4(0, 0, 0, 0);
                     int g = c_begin + rl;
@@ -290,22 +340,8 @@ k_gemv_fast(const DeviceTables* __restrict__ tab, const Problem* __restrict__ pr
                             n0 = __ldg(rec); n1 = __ldg(rec + B); n2 = __ldg(rec + 2 * size_t(B));
                         }
                         float v[8];
-                        v[0] = block_value<false>(sm_tab, a.x, h.x, X, xq_col);
-                        v[1] = block_value<true>(sm_tab, a.y, h.x, X, xq_col);
-                        v[2] = block_value<false>(sm_tab, a.z, h.y, X, xq_col);
-                        v[3] = block_value<true>(sm_tab, a.w, h.y, X, xq_col);
-                        v[4] = block_value<false>(sm_tab, b.x, h.z, X, xq_col);
-                        v[5] = block_value<true>(sm_tab, b.y, h.z, X, xq_col);
-                        v[6] = block_value<false>(sm_tab, b.z, h.w, X, xq_col);
-                        v[7] = block_value<true>(sm_tab, b.w, h.w, X, xq_col);
-                        // transpose through shared memory: lane l then owns row l/4, lanes 8(l%4)..8(l%4)+7
-                        __syncwarp();
-#pragma unroll
-                        for (int r = 0; r < 8; ++r) red[r * kRedStride + lane] = v[r];
-                        __syncwarp();
-                        const float4 s0 = *reinterpret_cast<const float4*>(red + (lane >> 2) * kRedStride + 8 * (lane & 3));
-                        const float4 s1 = *reinterpret_cast<const float4*>(red + (lane >> 2) * kRedStride + 8 * (lane & 3) + 4);
-                        float sum = ((s0.x + s0.y) + (s0.z + s0.w)) + ((s1.x + s1.y) + (s1.z + s1.w));
+                        record_values(sm_tab, a, b, h, X, xq_rec, v);
+                        float sum = transpose_partial(red, lane, v);
                         sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
                         sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
                         if ((lane & 3) == 0) rowacc[cg * rows_chunk + (g - c_begin) * 8 + (lane >> 2)] = sum;
@@ -331,30 +367,218 @@ k_gemv_fast(const DeviceTables* __restrict__ tab, const Problem* __restrict__ pr
     }
 }
 
-cudaError_t launch_gemv_fast(const Problem& single, int batch, const Problem* problems_dev, int count, int max_blocks,
-                             const void* table, cudaStream_t s) {
-    static int num_sms[64] = {0};
+static cudaError_t device_sms(int* sms) {
+    static int cached[64] = {0};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 64 && num_sms[dev] == 0) {
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (cached[dev] == 0) {
         int n = 0;
         e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(k_gemv_fast, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
-        num_sms[dev] = n;
+        cached[dev] = n;
     }
-    const int sms = dev < 64 ? num_sms[dev] : 148;
+    *sms = cached[dev];
+    return cudaSuccess;
+}
+
+cudaError_t launch_gemv_fast(const Problem& single, int batch, int max_blocks, const void* table, cudaStream_t s) {
+    int sms = 0;
+    cudaError_t e = device_sms(&sms);
+    if (e != cudaSuccess) return e;
     const FastSmemLayout L = fast_smem_layout(max_blocks);
     if (L.total > 227u * 1024u) return cudaErrorInvalidValue;
-    int grid = sms;
-    if (!problems_dev) {
-        const int groups = (single.N + 7) / 8;
-        if (groups < grid) grid = groups;
+    const int groups = (single.N + 7) / 8;
+    const int grid = groups < sms ? groups : sms;
+    k_gemv_fast<<<grid, kFastThreads, L.total, s>>>(static_cast<const DeviceTables*>(table), single, batch,
+                                                    max_blocks);
+    return cudaGetLastError();
+}
+
+// ===========================================================================
+// Planned list of matrices: k_prepare_x + k_gemv_units
+// ===========================================================================
+// Workspace written by grouped_plan (host) and read by both kernels:
+//   PlanHeader | Problem[count] | unit_prefix[count + 1] | col_prefix[count + 1] | pad | xq records
+struct PlanHeader {
+    int32_t count;
+    int32_t total_units;  // sum over matrices of ceil(N / 8)
+    int32_t total_cols;   // sum over matrices of words per row
+    int32_t reserved;
+    uint32_t off_problems, off_unit_prefix, off_col_prefix, off_xq;
+};
+
+static size_t plan_meta_bytes(int count) {
+    size_t b = sizeof(PlanHeader) + size_t(count) * sizeof(Problem) + 2 * size_t(count + 1) * 4;
+    return (b + 255) & ~size_t(255);
+}
+
+static inline int problem_blocks(const Problem& q) {
+    return (q.tail || q.K % 24 == 0) ? q.K / 24 : (q.K + 23) / 24;
+}
+
+size_t grouped_workspace_bytes(const Problem* problems, int count) {
+    size_t cols = 0;
+    for (int i = 0; i < count; ++i) cols += size_t(problem_blocks(problems[i]));
+    return plan_meta_bytes(count) + cols * kXqBytesPerCol;
+}
+
+// Largest p with prefix[p] <= v (prefix[0] = 0, prefix[count] > v).
+__device__ __forceinline__ int find_problem(const int32_t* __restrict__ prefix, int count, int v) {
+    int lo = 0, hi = count;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(prefix + mid) <= v) lo = mid; else hi = mid;
     }
-    k_gemv_fast<<<grid, kFastThreads, L.total, s>>>(static_cast<const DeviceTables*>(table), problems_dev, single,
-                                                    count, batch, max_blocks);
+    return lo;
+}
+
+__global__ void __launch_bounds__(256) k_prepare_x(unsigned char* __restrict__ ws) {
+    const PlanHeader* H = reinterpret_cast<const PlanHeader*>(ws);
+    const Problem* problems = reinterpret_cast<const Problem*>(ws + H->off_problems);
+    const int32_t* col_prefix = reinterpret_cast<const int32_t*>(ws + H->off_col_prefix);
+    uint4* xq = reinterpret_cast<uint4*>(ws + H->off_xq);
+    for (int gc = blockIdx.x * blockDim.x + threadIdx.x; gc < H->total_cols; gc += gridDim.x * blockDim.x) {
+        const int p = find_problem(col_prefix, H->count, gc);
+        const Problem P = problems[p];
+        uint32_t q[20];
+        quantise_column(static_cast<const __half*>(P.x), P.K, gc - col_prefix[p], q);
+#pragma unroll
+        for (int k = 0; k < 5; ++k) xq[size_t(gc) * 5 + k] = make_uint4(q[4 * k], q[4 * k + 1], q[4 * k + 2], q[4 * k + 3]);
+    }
+}
+
+__global__ void __launch_bounds__(kFastThreads, 1)
+k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restrict__ ws) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    unsigned char* smem = stage_fast_tables(tab, smem_raw);
+    const uint32_t sm_tab = smem_u32(smem);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float* red = reinterpret_cast<float*>(smem + kFastBytes) + warp * kRedFloats;
+    __syncthreads();  // the only CTA-wide barrier: tables are staged
+
+    const PlanHeader* H = reinterpret_cast<const PlanHeader*>(ws);
+    const Problem* problems = reinterpret_cast<const Problem*>(ws + H->off_problems);
+    const int32_t* unit_prefix = reinterpret_cast<const int32_t*>(ws + H->off_unit_prefix);
+    const int32_t* col_prefix = reinterpret_cast<const int32_t*>(ws + H->off_col_prefix);
+    const unsigned char* xq_all = ws + H->off_xq;
+    const int count = H->count, total_units = H->total_units;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+
+    // consecutive units (neighbouring row groups of a matrix) go to consecutive warps of the grid
+    for (int u = blockIdx.x * kFastWarps + warp; u < total_units; u += gridDim.x * kFastWarps) {
+        const int p = find_problem(unit_prefix, count, u);
+        const int g = u - __ldg(unit_prefix + p);
+        const Problem P = problems[p];
+        const int ntail = P.tail ? P.K % 24 : 0;
+        const int B = P.tail ? P.K / 24 : (P.K + 23) / 24;
+        const int CG = (B + 31) / 32;
+        const unsigned char* xq_p = xq_all + size_t(__ldg(col_prefix + p)) * kXqBytesPerCol;
+        const uint4* codes = static_cast<const uint4*>(P.codes) + size_t(g) * 3 * B;
+
+        float acc[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) acc[r] = 0.f;
+        uint4 n0 = zero4, n1 = zero4, n2 = zero4;
+        if (lane < B) {
+            n0 = __ldg(codes + lane); n1 = __ldg(codes + B + lane); n2 = __ldg(codes + 2 * size_t(B) + lane);
+        }
+        for (int cg = 0; cg < CG; ++cg) {
+            const int col = cg * 32 + lane;
+            const bool active = col < B;
+            const uint4 a = n0, b = n1, h = n2;
+            if (col + 32 < B) {  // prefetch the next column group's record
+                n0 = __ldg(codes + col + 32); n1 = __ldg(codes + B + col + 32);
+                n2 = __ldg(codes + 2 * size_t(B) + col + 32);
+            } else {
+                n0 = n1 = n2 = zero4;
+            }
+            const unsigned char* xq_rec = xq_p + size_t(active ? col : 0) * kXqBytesPerCol;
+            LaneX X;
+            {
+                uint32_t q[20];
+                const uint4* src = reinterpret_cast<const uint4*>(xq_rec);
+#pragma unroll
+                for (int k = 0; k < 5; ++k) {
+                    const uint4 t = __ldg(src + k);
+                    q[4 * k] = t.x; q[4 * k + 1] = t.y; q[4 * k + 2] = t.z; q[4 * k + 3] = t.w;
+                }
+                lane_x_from_words(q, active, X);
+            }
+            float v[8];
+            record_values(sm_tab, active ? a : zero4, active ? b : zero4, active ? h : zero4, X, xq_rec, v);
+#pragma unroll
+            for (int r = 0; r < 8; ++r) acc[r] += v[r];
+        }
+        // row sums, row scale, tail (Sec. 5.1); four lanes per row share the tail
+        float sum = transpose_partial(red, lane, acc);
+        const int row = g * 8 + (lane >> 2);
+        if (row < P.N) {
+            sum *= __ldg(P.row_scales + row);
+            const __half* xh = static_cast<const __half*>(P.x) + 24 * B;
+            const __half* tl = static_cast<const __half*>(P.tail) + size_t(row) * ntail;
+            for (int k = lane & 3; k < ntail; k += 4) sum = fmaf(__half2float(tl[k]), __half2float(xh[k]), sum);
+        }
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
+        if (row < P.N && (lane & 3) == 0) P.y[row] = sum;
+    }
+}
+
+cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, size_t ws_bytes, cudaStream_t s) {
+    const size_t meta = plan_meta_bytes(count);
+    if (ws_bytes < grouped_workspace_bytes(problems_host, count)) return cudaErrorInvalidValue;
+    unsigned char* buf = static_cast<unsigned char*>(calloc(1, meta));
+    if (!buf) return cudaErrorMemoryAllocation;
+    PlanHeader* H = reinterpret_cast<PlanHeader*>(buf);
+    H->count = count;
+    H->off_problems = uint32_t(sizeof(PlanHeader));
+    H->off_unit_prefix = H->off_problems + uint32_t(count) * uint32_t(sizeof(Problem));
+    H->off_col_prefix = H->off_unit_prefix + uint32_t(count + 1) * 4u;
+    H->off_xq = uint32_t(meta);
+    memcpy(buf + H->off_problems, problems_host, size_t(count) * sizeof(Problem));
+    int32_t* up = reinterpret_cast<int32_t*>(buf + H->off_unit_prefix);
+    int32_t* cp = reinterpret_cast<int32_t*>(buf + H->off_col_prefix);
+    long long units = 0, cols = 0;
+    for (int i = 0; i < count; ++i) {
+        up[i] = int32_t(units);
+        cp[i] = int32_t(cols);
+        units += (problems_host[i].N + 7) / 8;
+        cols += problem_blocks(problems_host[i]);
+    }
+    up[count] = int32_t(units);
+    cp[count] = int32_t(cols);
+    cudaError_t e = cudaSuccess;
+    if (units > 0x7FFFFFF0LL || cols > 0x7FFFFFF0LL) e = cudaErrorInvalidValue;
+    H->total_units = int32_t(units);
+    H->total_cols = int32_t(cols);
+    // pageable source: the runtime stages it before returning, so the buffer can be freed
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ws_dev, buf, meta, cudaMemcpyHostToDevice, s);
+    free(buf);
+    return e;
+}
+
+cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s) {
+    int sms = 0;
+    cudaError_t e = device_sms(&sms);
+    if (e != cudaSuccess) return e;
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const uint32_t smem = kTableSmemBytes + kFastWarps * kRedFloats * 4;
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(k_gemv_units, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    k_prepare_x<<<sms * 2, 256, 0, s>>>(static_cast<unsigned char*>(ws_dev));
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    k_gemv_units<<<sms, kFastThreads, smem, s>>>(static_cast<const DeviceTables*>(table),
+                                                 static_cast<const unsigned char*>(ws_dev));
     return cudaGetLastError();
 }
 

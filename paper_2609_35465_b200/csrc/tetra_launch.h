@@ -28,10 +28,14 @@ cudaError_t launch_decode_packed(const void* packed, const void* table, int8_t* 
 cudaError_t launch_gemv_paper(const void* codes, size_t row_stride, const float* row_scales, const void* table,
                               const void* x, float* y, int N, int K, int batch, const void* tail, cudaStream_t s);
 
-// Fast GEMV.  `problems_dev` == nullptr: one product described by `single`
-// (x and y advanced per batch column inside).  Otherwise `count` products read
-// from device memory, batch 1 each.
-cudaError_t launch_gemv_fast(const Problem& single, int batch, const Problem* problems_dev, int count, int max_blocks,
-                             const void* table, cudaStream_t s);
+// Fast GEMV of one matrix (x and y advanced per batch column inside); no scratch memory.
+cudaError_t launch_gemv_fast(const Problem& single, int batch, int max_blocks, const void* table, cudaStream_t s);
+
+// Planned list of batch-1 products.  grouped_plan writes descriptors and prefix
+// arrays to the workspace (once per list); grouped_run enqueues the activation
+// pre-pass and the persistent GEMV kernel (every step).
+size_t grouped_workspace_bytes(const Problem* problems_host, int count);
+cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, size_t ws_bytes, cudaStream_t s);
+cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s);
 
 }  // namespace tetra

@@ -17,7 +17,7 @@ struct PaperTables {
 static_assert(sizeof(PaperTables) == 18816, "paper table blob is 18,816 bytes");
 
 constexpr uint32_t kTableMagic = 0x54455442u;  // "TETB"
-constexpr uint32_t kTableVersion = 3;
+constexpr uint32_t kTableVersion = 4;
 constexpr int kMiddleClass0 = 1240;            // N0 of Sec. 3.3 (checked at build)
 
 // Everything tetra_build_table copies to the device, in one blob.
@@ -29,14 +29,16 @@ struct DeviceTables {
     // ---- fast path: everything below is staged in shared memory ------------
     // Rank rows for PRMT lookup: nibble j = rank (0..3); a coordinate of rank 4
     // is stored as 8 | 2 (bit 3 flags it for the fix-up path).
-    uint32_t rows_fast[4096];   // 18832
-    uint32_t mid_fast[2048];    // 35216: rows_fast[mix(i2)], indexed by i2 directly
+    // (the kernels place this part on a 16 KiB boundary of shared memory, so each
+    //  sub-table's offset can be OR-ed into an index instead of added)
+    uint32_t rows_fast[4096];   // +0
+    uint32_t mid_fast[2048];    // +16384: rows_fast[mix(i2)], indexed by i2 directly
+    float scale[2][32];         // +24576: gain[g] / sqrt(16 m)
     // Pattern-byte masks of the Turyn coordinates: bit 4j+2 set where the
     // Hamming word has coordinate j set; H for a and b, H' for x.
-    uint32_t mask_h[16];        // 43408
-    uint32_t mask_hr[16];       // 43472
-    float scale[2][32];         // 43536: gain[g] / sqrt(16 m)
-    uint32_t pad_[16];          // 43792 (spare)
+    uint32_t mask_h[16];        // +24832
+    uint32_t mask_hr[16];       // +24896
+    uint32_t pad_[16];          // +24960 (spare)
     // ---- pack-time only (global memory) ------------------------------------
     // 12 trellis bits (s8 | b1<<6 | b2<<7 | b3<<11) -> Turyn coordinates a | b<<4 | x<<8.
     uint16_t trellis_to_abx[4096];

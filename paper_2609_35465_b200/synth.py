@@ -103,3 +103,30 @@ def tails(seed: int, stream: int, sigma: np.ndarray, ntail: int) -> np.ndarray:
 # 24 dimensions; the paper does not print its two gain values, and both the
 # oracle and the CUDA path simply read whatever pair they are given.
 DEFAULT_GAIN = np.array([4.3156, 5.4415], dtype=np.float32)
+
+
+# ---------------------------------------------------------------------------
+# The same code stream generated with torch ops (on any device), for workloads
+# too large to draw on the host in reasonable time.  Bit-identical to codes().
+# ---------------------------------------------------------------------------
+def _s64(v: int) -> int:
+    v &= 0xFFFFFFFFFFFFFFFF
+    return v - (1 << 64) if v >= (1 << 63) else v
+
+
+def codes_torch(seed: int, stream: int, N: int, B: int, device="cpu"):
+    """File-order codes uint8 [N, B, 6] as a torch tensor on `device`."""
+    import torch
+
+    def lsr(z, k):  # logical shift right of int64 bit patterns
+        return (z >> k) & ((1 << (64 - k)) - 1)
+
+    base = int(_stream_base(seed, stream, 0))
+    n = N * B
+    z = torch.arange(n, dtype=torch.int64, device=device) + _s64(base)
+    z = z + _s64(0x9E3779B97F4A7C15)
+    z = (z ^ lsr(z, 30)) * _s64(0xBF58476D1CE4E5B9)
+    z = (z ^ lsr(z, 27)) * _s64(0x94D049BB133111EB)
+    z = z ^ lsr(z, 31)
+    w = lsr(z, 16)
+    return w.view(torch.uint8).reshape(n, 8)[:, :6].contiguous().reshape(N, B, 6)

@@ -54,11 +54,14 @@ def lib():
         L.tetra_decode_packed.argtypes = [vp, vp, vp, vp, i32, i32, vp]
         L.tetra_gemv.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp]
         L.tetra_gemv_tail.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp]
-        L.tetra_grouped_workspace_bytes.argtypes = [i32]
+        L.tetra_grouped_workspace_bytes.argtypes = [vp, i32]
         L.tetra_grouped_workspace_bytes.restype = sz
+        L.tetra_gemv_grouped_plan.argtypes = [vp, i32, vp, sz, vp]
+        L.tetra_gemv_grouped_run.argtypes = [vp, vp, vp]
         L.tetra_gemv_grouped.argtypes = [vp, i32, vp, vp, sz, vp]
         L.tetra_gemv_paper_design.argtypes = [vp, sz, vp, vp, vp, vp, i32, i32, i32, vp, vp]
         L.tetra_gemv_hostio.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp]
+        L.tetra_gemv_grouped_hostio.argtypes = [vp, vp, vp, vp, sz, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -160,12 +163,23 @@ def make_problems(items):
     return arr
 
 
-def tetra_grouped_workspace_bytes(count: int) -> int:
-    return lib().tetra_grouped_workspace_bytes(count)
+def tetra_grouped_workspace_bytes(problems) -> int:
+    return lib().tetra_grouped_workspace_bytes(problems, len(problems))
+
+
+def tetra_gemv_grouped_plan(problems, workspace: torch.Tensor, stream=None):
+    """Writes the plan of a list of products (ctypes array from make_problems) into the workspace."""
+    _check(lib().tetra_gemv_grouped_plan(problems, len(problems), _ptr(workspace), workspace.numel(),
+                                         _stream(stream)), "tetra_gemv_grouped_plan")
+
+
+def tetra_gemv_grouped_run(workspace: torch.Tensor, table, stream=None):
+    """One step of a planned list: activation pre-pass + persistent GEMV kernel."""
+    _check(lib().tetra_gemv_grouped_run(_ptr(workspace), _ptr(table), _stream(stream)), "tetra_gemv_grouped_run")
 
 
 def tetra_gemv_grouped(problems, table, workspace: torch.Tensor, stream=None):
-    """problems: ctypes array from make_problems; one persistent launch for all of them."""
+    """plan + run."""
     _check(lib().tetra_gemv_grouped(problems, len(problems), _ptr(table), _ptr(workspace), workspace.numel(),
                                     _stream(stream)), "tetra_gemv_grouped")
 
@@ -183,3 +197,11 @@ def tetra_gemv_hostio(codes, row_scales, table, x_host, y_host, x_stage, y_stage
     _check(lib().tetra_gemv_hostio(_ptr(codes), _ptr(row_scales), _ptr(table), _ptr(x_host), _ptr(y_host),
                                    _ptr(x_stage), _ptr(y_stage), N, K, batch, _ptr(tail), _stream(stream)),
            "tetra_gemv_hostio")
+
+
+def tetra_gemv_grouped_hostio(workspace, table, x_host, x_dev, y_host, y_dev, stream=None):
+    """A planned run with pinned host activations / results (one copy in, the kernels, one copy out)."""
+    _check(lib().tetra_gemv_grouped_hostio(_ptr(workspace), _ptr(table), _ptr(x_host), _ptr(x_dev),
+                                           x_dev.numel() * x_dev.element_size(), _ptr(y_host), _ptr(y_dev),
+                                           y_dev.numel() * y_dev.element_size(), _stream(stream)),
+           "tetra_gemv_grouped_hostio")

@@ -98,16 +98,21 @@ def test_grouped_launch_one_layer(tt, table, orc):
     mats = [make_matrix(34, i, mm.N, mm.K, True) for i, mm in enumerate(shapes.QWEN3_4B.layer_matrices())]
     devs = [upload(tt, table, m) for m in mats]
     problems = tt.make_problems(devs)
-    ws = torch.empty(tt.tetra_grouped_workspace_bytes(len(devs)), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(tt.tetra_grouped_workspace_bytes(problems), dtype=torch.uint8, device="cuda")
     tt.tetra_gemv_grouped(problems, table, ws)
     torch.cuda.synchronize()
-    for m, d in zip(mats, devs):
+    first = [d["y"].cpu().numpy().copy() for d in devs]
+    tt.tetra_gemv_grouped_run(ws, table)                   # the plan can be run again: same bits
+    torch.cuda.synchronize()
+    for m, d, f in zip(mats, devs, first):
         y = d["y"].cpu().numpy()[0]
+        assert np.array_equal(y, f[0])
         assert_gemv_close(y, oracle_product(orc, m, GAIN), "grouped %dx%d" % (m["N"], m["K"]))
-        # same bits as the single-matrix entry point (the reduction order is fixed)
+        # the single-matrix entry point sums in another order: equal up to float32 rounding
         d["y"].fill_(float("nan"))
         y1 = run_fast(tt, table, m, d)[0]
-        assert np.array_equal(y, y1)
+        assert np.linalg.norm(y - y1) <= 1e-5 * np.linalg.norm(y)
+
 
 
 def test_special_inputs(tt, table, orc):
