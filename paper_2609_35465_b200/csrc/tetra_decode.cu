@@ -71,14 +71,14 @@ __device__ __forceinline__ void emit_block(const FastBlock& fb, int8_t* __restri
     for (int k = 0; k < 6; ++k)
 #pragma unroll
         for (int i = 0; i < 4; ++i) y[4 * k + i] = int(int8_t((fb.y0[k] >> (8 * i)) & 0xFF));
-    if (fb.flags1) {
+    if (fb.row1 & kRank4Flags) {
         int j, dy, dsq;
-        rank4_fix(fb.flags1, fb.sel1, &j, &dy, &dsq);
+        rank4_fix(fb.row1 & kRank4Flags, fb.sel1, &j, &dy, &dsq);
         y[j] += dy;
     }
-    if (fb.flags3) {
+    if (fb.row3 & kRank4Flags) {
         int j, dy, dsq;
-        rank4_fix(fb.flags3, fb.sel3, &j, &dy, &dsq);
+        rank4_fix(fb.row3 & kRank4Flags, fb.sel3, &j, &dy, &dsq);
         y[16 + j] += dy;
     }
     int norm = 0;

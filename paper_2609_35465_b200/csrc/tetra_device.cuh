@@ -150,8 +150,8 @@ constexpr uint32_t kRank4Flags = 0x88888888u;
 
 struct FastBlock {
     uint32_t y0[6];   // p = 0 image, int8 x 4, coordinate 4k+i in byte i of y0[k]
-    uint32_t flags1;  // row1 & 0x88888888: the rank-4 coordinate of section 1, if any
-    uint32_t flags3;  // same for section 3
+    uint32_t row1;    // rank rows of sections 1 and 3 (bit 3 of a nibble flags a rank-4 coordinate)
+    uint32_t row3;
     uint32_t sel1;    // PRMT selectors (rank | c << 2 per nibble), for the fix-up
     uint32_t sel3;
     uint32_t p13;     // p << 13
@@ -196,8 +196,8 @@ __device__ __forceinline__ void fast_decode(uint32_t sm_tab, uint32_t w0, uint32
     out.y0[3] = prmt(kPoolLo, kPoolHi, sel2 >> 16);
     out.y0[4] = prmt(kPoolLo, kPoolHi, sel3);
     out.y0[5] = prmt(kPoolLo, kPoolHi, sel3 >> 16);
-    out.flags1 = row1 & kRank4Flags;
-    out.flags3 = row3 & kRank4Flags;
+    out.row1 = row1;
+    out.row3 = row3;
     out.sel1 = sel1;
     out.sel3 = sel3;
     out.p13 = (addr1 ^ addr3p) & 0x2000u;  // r ^ q = p

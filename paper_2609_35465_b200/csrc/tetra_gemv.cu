@@ -203,17 +203,17 @@ __device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint3
     }
     // |sum_j y_j q_j| <= sqrt(24 * 416) * 2^23 < 2^31: the block's dot product is an exact int32
     int dot = dh * 65536 + (dm * 256 + dl);
-    if (fb.flags1 | fb.flags3) {  // a coordinate of rank 4: about 1.6 % of uniform random words
-        if (fb.flags1) {
+    if ((fb.row1 | fb.row3) & kRank4Flags) {  // a coordinate of rank 4: about 1.6 % of uniform random words
+        if (fb.row1 & kRank4Flags) {
             int j, dy, dsq;
-            rank4_fix(fb.flags1, fb.sel1, &j, &dy, &dsq);
+            rank4_fix(fb.row1 & kRank4Flags, fb.sel1, &j, &dy, &dsq);
             dot += dy * xq_coord(xq_rec, j);
             n2 += dsq;
             n1 += dy;
         }
-        if (fb.flags3) {
+        if (fb.row3 & kRank4Flags) {
             int j, dy, dsq;
-            rank4_fix(fb.flags3, fb.sel3, &j, &dy, &dsq);
+            rank4_fix(fb.row3 & kRank4Flags, fb.sel3, &j, &dy, &dsq);
             dot += dy * xq_coord(xq_rec, 16 + j);
             n2 += dsq;
             n1 += dy;
@@ -466,8 +466,6 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
     const int32_t* col_prefix = reinterpret_cast<const int32_t*>(ws + H->off_col_prefix);
     const unsigned char* xq_all = ws + H->off_xq;
     const int count = H->count, total_units = H->total_units;
-    const uint4 zero4 = make_uint4(0, 0, 0, 0);
-
     // consecutive units (neighbouring row groups of a matrix) go to consecutive warps of the grid
     for (int u = blockIdx.x * kFastWarps + warp; u < total_units; u += gridDim.x * kFastWarps) {
         const int p = find_problem(unit_prefix, count, u);
@@ -482,34 +480,31 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
         float acc[8];
 #pragma unroll
         for (int r = 0; r < 8; ++r) acc[r] = 0.f;
-        uint4 n0 = zero4, n1 = zero4, n2 = zero4;
-        if (lane < B) {
-            n0 = __ldg(codes + lane); n1 = __ldg(codes + B + lane); n2 = __ldg(codes + 2 * size_t(B) + lane);
-        }
+        // lanes beyond the last column re-read column B - 1 and contribute with a zero step
+        const uint32_t Bu = uint32_t(B);
+        uint32_t col = min(uint32_t(lane), Bu - 1);
+        uint4 n0 = __ldg(codes + col), n1 = __ldg(codes + Bu + col), n2 = __ldg(codes + 2 * Bu + col);
         for (int cg = 0; cg < CG; ++cg) {
-            const int col = cg * 32 + lane;
-            const bool active = col < B;
+            const bool active = uint32_t(cg * 32 + lane) < Bu;
             const uint4 a = n0, b = n1, h = n2;
-            if (col + 32 < B) {  // prefetch the next column group's record
-                n0 = __ldg(codes + col + 32); n1 = __ldg(codes + B + col + 32);
-                n2 = __ldg(codes + 2 * size_t(B) + col + 32);
-            } else {
-                n0 = n1 = n2 = zero4;
+            const unsigned char* xq_rec = xq_p + col * uint32_t(kXqBytesPerCol);
+            col = min(uint32_t((cg + 1) * 32 + lane), Bu - 1);
+            if (cg + 1 < CG) {  // prefetch the next column group's record
+                n0 = __ldg(codes + col); n1 = __ldg(codes + Bu + col); n2 = __ldg(codes + 2 * Bu + col);
             }
-            const unsigned char* xq_rec = xq_p + size_t(active ? col : 0) * kXqBytesPerCol;
             LaneX X;
             {
-                uint32_t q[20];
                 const uint4* src = reinterpret_cast<const uint4*>(xq_rec);
-#pragma unroll
-                for (int k = 0; k < 5; ++k) {
-                    const uint4 t = __ldg(src + k);
-                    q[4 * k] = t.x; q[4 * k + 1] = t.y; q[4 * k + 2] = t.z; q[4 * k + 3] = t.w;
-                }
-                lane_x_from_words(q, active, X);
+                const uint4 t0 = __ldg(src), t1 = __ldg(src + 1), t2 = __ldg(src + 2), t3 = __ldg(src + 3),
+                            t4 = __ldg(src + 4);
+                X.hi[0] = t0.x; X.hi[1] = t0.y; X.hi[2] = t0.z; X.hi[3] = t0.w; X.hi[4] = t1.x; X.hi[5] = t1.y;
+                X.mid[0] = t1.z; X.mid[1] = t1.w; X.mid[2] = t2.x; X.mid[3] = t2.y; X.mid[4] = t2.z; X.mid[5] = t2.w;
+                X.lo[0] = t3.x; X.lo[1] = t3.y; X.lo[2] = t3.z; X.lo[3] = t3.w; X.lo[4] = t4.x; X.lo[5] = t4.y;
+                X.step = active ? __uint_as_float(t4.z) : 0.f;
+                X.sum = int(t4.w);
             }
             float v[8];
-            record_values(sm_tab, active ? a : zero4, active ? b : zero4, active ? h : zero4, X, xq_rec, v);
+            record_values(sm_tab, a, b, h, X, xq_rec, v);
 #pragma unroll
             for (int r = 0; r < 8; ++r) acc[r] += v[r];
         }
