@@ -47,7 +47,8 @@ enum {
     TETRA_BLOCK = 24,              /* weights per word */
     TETRA_WORD_BYTES = 6,
     TETRA_MAX_BATCH = 16,
-    TETRA_PAPER_TABLE_BYTES = 18816 /* 16384 + 2304 + 128, Sec. 3.4 */
+    TETRA_PAPER_TABLE_BYTES = 18816, /* 16384 + 2304 + 128, Sec. 3.4 */
+    TETRA_NOALLOC_MAX_K = 24576      /* largest K tetra_gemv_noalloc accepts */
 };
 
 /* Human-readable name of a status code (static storage). */
@@ -172,6 +173,27 @@ int tetra_gemv_hostio(const void *codes, const float *row_scales, const void *ta
 int tetra_gemv_grouped_hostio(void *workspace_dev, const void *table, const void *x_host,
                               void *x_dev, size_t x_bytes, float *y_host, const float *y_dev,
                               size_t y_bytes, void *stream);
+
+/* The batch-1 product of tetra_gemv_tail for callers that cannot allocate
+ * device memory (the paper has no counterpart: this is a packaging of the same
+ * kernels).  A plug-in inside an application that owns the GPU's memory pool, a
+ * control loop that may not touch the allocator, a process with a fixed memory
+ * budget: none of them can hand the planned-list kernels the scratch buffer
+ * they need, so this entry point keeps that buffer inside the library, as a
+ * fixed array of 82,176 bytes in its device image (held by every GPU that
+ * loads the library, until the process exits).  The call itself allocates
+ * nothing, on the host or on the device.
+ *   - Arguments as tetra_gemv_tail with batch = 1; tail == NULL selects the
+ *     zero-pad rule.  K > TETRA_NOALLOC_MAX_K returns TETRA_ERR_SIZE.
+ *   - The first call on a device looks up the array's device address; make
+ *     that call before any stream capture begins on that device.
+ *   - All calls share the one array, which keeps whatever the last call wrote.
+ *     Nothing in it needs clearing (each call rewrites all it reads), but two
+ *     calls that run on the GPU at the same time, on any streams, race on it:
+ *     keep calls on one device in stream order, or serialise them.
+ *   - Enqueues one small copy and two kernels on `stream`; does not synchronise. */
+int tetra_gemv_noalloc(const void *codes, const float *row_scales, const void *table,
+                       const void *x, float *y, int N, int K, const void *tail, void *stream);
 
 #ifdef __cplusplus
 }

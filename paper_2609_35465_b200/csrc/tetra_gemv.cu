@@ -556,6 +556,29 @@ cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, 
     return e;
 }
 
+size_t single_plan_meta_bytes() { return plan_meta_bytes(1); }
+
+size_t single_plan_scratch_bytes(int blocks_per_row) {
+    return plan_meta_bytes(1) + size_t(blocks_per_row) * kXqBytesPerCol;
+}
+
+void single_plan_fill(const Problem& problem, unsigned char* meta_host) {
+    memset(meta_host, 0, plan_meta_bytes(1));
+    PlanHeader* H = reinterpret_cast<PlanHeader*>(meta_host);
+    H->count = 1;
+    H->total_units = (problem.N + 7) / 8;
+    H->total_cols = problem_blocks(problem);
+    H->off_problems = uint32_t(sizeof(PlanHeader));
+    H->off_unit_prefix = H->off_problems + uint32_t(sizeof(Problem));
+    H->off_col_prefix = H->off_unit_prefix + 8u;
+    H->off_xq = uint32_t(plan_meta_bytes(1));
+    memcpy(meta_host + H->off_problems, &problem, sizeof(Problem));
+    int32_t* up = reinterpret_cast<int32_t*>(meta_host + H->off_unit_prefix);
+    int32_t* cp = reinterpret_cast<int32_t*>(meta_host + H->off_col_prefix);
+    up[0] = 0; up[1] = H->total_units;
+    cp[0] = 0; cp[1] = H->total_cols;
+}
+
 cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s) {
     int sms = 0;
     cudaError_t e = device_sms(&sms);

@@ -38,4 +38,13 @@ size_t grouped_workspace_bytes(const Problem* problems_host, int count);
 cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, size_t ws_bytes, cudaStream_t s);
 cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s);
 
+
+// Plan of a single product, for callers that bring their own scratch memory:
+// single_plan_fill writes single_plan_meta_bytes() bytes of plan data to a host
+// buffer; copied to the start of a scratch area of single_plan_scratch_bytes(blocks)
+// bytes, it makes that area a valid argument of grouped_run.
+size_t single_plan_meta_bytes();
+size_t single_plan_scratch_bytes(int blocks_per_row);
+void single_plan_fill(const Problem& problem, unsigned char* meta_host);
+
 }  // namespace tetra

@@ -62,6 +62,7 @@ def lib():
         L.tetra_gemv_paper_design.argtypes = [vp, sz, vp, vp, vp, vp, i32, i32, i32, vp, vp]
         L.tetra_gemv_hostio.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp]
         L.tetra_gemv_grouped_hostio.argtypes = [vp, vp, vp, vp, sz, vp, vp, sz, vp]
+        L.tetra_gemv_noalloc.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, vp]
         _lib = L
     return _lib
 
@@ -205,3 +206,15 @@ def tetra_gemv_grouped_hostio(workspace, table, x_host, x_dev, y_host, y_dev, st
                                            x_dev.numel() * x_dev.element_size(), _ptr(y_host), _ptr(y_dev),
                                            y_dev.numel() * y_dev.element_size(), _stream(stream)),
            "tetra_gemv_grouped_hostio")
+
+
+NOALLOC_MAX_K = 24576
+
+
+def tetra_gemv_noalloc(codes, row_scales, table, x, y, N: int, K: int, tail=None, stream=None):
+    """Batch-1 product for callers that may not allocate device memory: the
+    scratch buffer lives inside the library (a fixed array, K <= NOALLOC_MAX_K).
+    Calls on one device share that array, so they must not overlap on the GPU."""
+    _check(lib().tetra_gemv_noalloc(_ptr(codes), _ptr(row_scales), _ptr(table), _ptr(x), _ptr(y), N, K,
+                                    _ptr(tail), _stream(stream)), "tetra_gemv_noalloc")
+    return y
