@@ -191,13 +191,13 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
-    if rank == 0:
+    if rank == 0 and not os.environ.get("TETRA_LIB"):
         tbuild.build()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
         dist.barrier()
-    elif not os.path.exists(tbuild.LIB):
+    elif not os.path.exists(tbuild.LIB) and not os.environ.get("TETRA_LIB"):
         tbuild.build()
 
     model = shapes.MODELS[args.model]

@@ -27,7 +27,7 @@ def _stale() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if not (force or _stale()):
         return LIB
-    flags = list(FLAGS)
+    flags = list(FLAGS) + os.environ.get("TETRA_EXTRA_FLAGS", "").split()
     if verbose:
         flags += ["-Xptxas", "-v"]
     objs = []

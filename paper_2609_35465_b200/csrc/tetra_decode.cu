@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(256) k_pack(const uint8_t* __restrict__ codes,
         for (int r = 0; r < 8; ++r) {
             const int row = 8 * G + r;
             const uint64_t w = row < N ? load_file_word(codes, size_t(row) * B + c) : 0ull;
-            file_to_device_word(w, tab->trellis_to_abx, &w0[r], &w1[r]);
+            file_to_device_word(w, tab, &w0[r], &w1[r]);
         }
         uint4* rec = packed + size_t(G) * 3 * B + c;
         rec[0] = make_uint4(w0[0], w0[1], w0[2], w0[3]);
@@ -70,23 +70,10 @@ __device__ __forceinline__ void emit_block(const FastBlock& fb, int8_t* __restri
 #pragma unroll
     for (int k = 0; k < 6; ++k)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) y[4 * k + i] = int(int8_t((fb.y0[k] >> (8 * i)) & 0xFF));
-    if (fb.row1 & kRank4Flags) {
-        int j, dy, dsq;
-        rank4_fix(fb.row1 & kRank4Flags, fb.sel1, &j, &dy, &dsq);
-        y[j] += dy;
-    }
-    if (fb.row3 & kRank4Flags) {
-        int j, dy, dsq;
-        rank4_fix(fb.row3 & kRank4Flags, fb.sel3, &j, &dy, &dsq);
-        y[16 + j] += dy;
-    }
+        for (int i = 0; i < 4; ++i) y[4 * k + i] = int(int8_t((fb.y[k] >> (8 * i)) & 0xFF));
     int norm = 0;
 #pragma unroll
-    for (int k = 0; k < 24; ++k) {
-        if (fb.p13) y[k] = 1 - y[k];
-        norm += y[k] * y[k];
-    }
+    for (int k = 0; k < 24; ++k) norm += y[k] * y[k];
     uint32_t* dst = reinterpret_cast<uint32_t*>(y_out + 24 * block);
 #pragma unroll
     for (int k = 0; k < 6; ++k)

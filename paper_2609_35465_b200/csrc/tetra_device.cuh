@@ -6,10 +6,12 @@
 //     tetra_decode_blocks and by the paper-design GEMV.
 //   * the fast decoder: works on the re-ordered 48-bit device word written by
 //     tetra_pack_codes and on tables staged in shared memory.  It produces the
-//     p = 0 image y0 of the lattice point as packed int8 (four coordinates per
-//     register, one PRMT per four); the true point is y0 when p = 0 and
-//     1 - y0 when p = 1 (shifting o = p + 2c by one maps every rank list of
-//     Sec. 3.3 onto one minus the list two places on).
+//     lattice point as packed int8, four coordinates per register and one PRMT
+//     per four: a selector nibble is rank | c << 2 and the 8-byte PRMT pool holds
+//     the rank lists of Sec. 3.3 for the block's parity p.  Branch-free: rows
+//     with a coordinate of rank 4 sit in the last 32 slots of their class, and
+//     for those slots two multiply-adds turn the pool's rank-2 entries into the
+//     rank-4 values.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -102,17 +104,22 @@ __device__ __forceinline__ void decode_file_word(const PaperTables* T, uint64_t 
 
 // ---------------------------------------------------------------------------
 // Device word (written by the pack kernel).  48 bits = w0 (32) + w1 (16):
-//   w0: [0..10] i1  [11] r  [12..22] i3  [23] q = p^r  [24..27] a  [28..31] b
+//   w0: [0..10] i1'  [11] r  [12..22] i3'  [23] q = p^r  [24..27] a  [28..31] b
 //   w1: [0..10] i2  [11..14] x  [15] g
-// (a, b, x) are the Turyn coordinates of the trellis path: the three pattern
-// bytes are h(a)+h'(x), h(b)+h'(x), h(a)+h(b)+h'(x).
+// i1', i3' are the row indices after the per-class permutation row_perm (class r
+// for section 1, class r3 = p^r^delta for section 3).  (a, b, x) are the Turyn
+// coordinates of the trellis path: the three pattern bytes are h(a)+h'(x),
+// h(b)+h'(x), h(a)+h(b)+h'(x).
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ void file_to_device_word(uint64_t w, const uint16_t* trellis_to_abx,
-                                                    uint32_t* w0, uint32_t* w1) {
-    const uint32_t i1 = uint32_t(w & 0x7FF), i2 = uint32_t((w >> 11) & 0x7FF), i3 = uint32_t((w >> 22) & 0x7FF);
+__device__ __forceinline__ void file_to_device_word(uint64_t w, const DeviceTables* tab, uint32_t* w0, uint32_t* w1) {
+    uint32_t i1 = uint32_t(w & 0x7FF), i3 = uint32_t((w >> 22) & 0x7FF);
+    const uint32_t i2 = uint32_t((w >> 11) & 0x7FF);
     const uint32_t path = uint32_t((w >> 33) & 0xFFF);
     const uint32_t p = uint32_t((w >> 45) & 1), r = uint32_t((w >> 46) & 1), g = uint32_t((w >> 47) & 1);
-    const uint32_t abx = trellis_to_abx[path];
+    const uint32_t r3 = p ^ r ^ uint32_t(i2 >= uint32_t(kMiddleClass0));  // Eq. (3)
+    i1 = tab->row_perm[r][i1];
+    i3 = tab->row_perm[r3][i3];
+    const uint32_t abx = tab->trellis_to_abx[path];
     *w0 = i1 | (r << 11) | (i3 << 12) | ((p ^ r) << 23) | ((abx & 0xFFu) << 24);
     *w1 = i2 | ((abx >> 8) << 11) | (g << 15);
 }
@@ -142,21 +149,27 @@ __device__ __forceinline__ unsigned char* stage_fast_tables(const DeviceTables* 
 }
 constexpr uint32_t kTableSmemBytes = uint32_t(kFastBytes) + kSmAlign;
 
-// PRMT pool of the p = 0 image, indexed by rank | c << 2:
-//   c = 0: 0, 4, -4, 8     c = 1: 2, -2, 6, -6
-constexpr uint32_t kPoolLo = 0x08FC0400u;
-constexpr uint32_t kPoolHi = 0xFA06FE02u;
-constexpr uint32_t kRank4Flags = 0x88888888u;
+// PRMT pools, indexed by rank | c << 2 (ranks 0..3 of the lists of Sec. 3.3):
+//   p = 0:  c = 0: 0, 4, -4, 8     c = 1: 2, -2, 6, -6
+//   p = 1:  c = 0: 1, -3, 5, -7    c = 1: -1, 3, -5, 7
+// The rank-4 values differ from the rank-2 ones (entries 2 and 6, byte 2 of each
+// word) by 4 s and -4 s with s = 2p - 1:  -8, 10 for p = 0;  9, -9 for p = 1.  Adding
+// +-(4 << 16) to the two words never carries out of byte 2.
+constexpr uint32_t kPool0Lo = 0x08FC0400u, kPool0Hi = 0xFA06FE02u;
+constexpr uint32_t kPool1Lo = 0xF905FD01u, kPool1Hi = 0x07FB03FFu;
+constexpr uint32_t kRank4Step = 4u << 16;
 
 struct FastBlock {
-    uint32_t y0[6];   // p = 0 image, int8 x 4, coordinate 4k+i in byte i of y0[k]
-    uint32_t row1;    // rank rows of sections 1 and 3 (bit 3 of a nibble flags a rank-4 coordinate)
-    uint32_t row3;
-    uint32_t sel1;    // PRMT selectors (rank | c << 2 per nibble), for the fix-up
-    uint32_t sel3;
-    uint32_t p13;     // p << 13
-    uint32_t goff;    // shared-memory address of the gain's half of the scale table (bit 7 = g)
+    uint32_t y[6];  // the lattice point, int8 x 4, coordinate 4k+i in byte i of y[k]
+    uint32_t goff;  // shared-memory address of the gain's half of the scale table (bit 7 = g)
 };
+
+// 1 if the 11-bit row index in the top bits of `x` lies in the last 32 slots of its class.
+__device__ __forceinline__ uint32_t top_slots_flag(uint32_t x) {
+    uint32_t f;
+    asm("{ .reg .u32 t; add.cc.u32 t, %1, %2; addc.u32 %0, 0, 0; }" : "=r"(f) : "r"(x), "r"(uint32_t(kRank4Slots) << 21));
+    return f;
+}
 
 // HI = false: w1 sits in bits 0..15 of `w1pair`; HI = true: in bits 16..31.
 // sm_tab: shared-memory address of the staged tables, a multiple of 16 KiB, so
@@ -164,8 +177,8 @@ struct FastBlock {
 // masks it.
 template <bool HI>
 __device__ __forceinline__ void fast_decode(uint32_t sm_tab, uint32_t w0, uint32_t w1pair, FastBlock& out) {
-    const uint32_t addr1 = ((w0 << 2) & 0x3FFCu) | (sm_tab + kSmRows);    // (i1 | r << 11) * 4
-    const uint32_t addr3p = ((w0 >> 10) & 0x3FFCu) | (sm_tab + kSmRows);  // (i3 | q << 11) * 4
+    const uint32_t addr1 = ((w0 << 2) & 0x3FFCu) | (sm_tab + kSmRows);    // (i1' | r << 11) * 4
+    const uint32_t addr3p = ((w0 >> 10) & 0x3FFCu) | (sm_tab + kSmRows);  // (i3' | q << 11) * 4
     const uint32_t a4 = ((w0 >> 22) & 0x3Cu) | (sm_tab + kSmMaskH);
     const uint32_t b4 = ((w0 >> 26) & 0x3Cu) | (sm_tab + kSmMaskH);
     uint32_t addr2, x4;
@@ -190,29 +203,22 @@ __device__ __forceinline__ void fast_decode(uint32_t sm_tab, uint32_t w0, uint32
     const uint32_t sel1 = row1 ^ ma ^ mx;
     const uint32_t sel2 = row2 ^ mb ^ mx;
     const uint32_t sel3 = row3 ^ (ma ^ mb) ^ mx;
-    out.y0[0] = prmt(kPoolLo, kPoolHi, sel1);
-    out.y0[1] = prmt(kPoolLo, kPoolHi, sel1 >> 16);
-    out.y0[2] = prmt(kPoolLo, kPoolHi, sel2);
-    out.y0[3] = prmt(kPoolLo, kPoolHi, sel2 >> 16);
-    out.y0[4] = prmt(kPoolLo, kPoolHi, sel3);
-    out.y0[5] = prmt(kPoolLo, kPoolHi, sel3 >> 16);
-    out.row1 = row1;
-    out.row3 = row3;
-    out.sel1 = sel1;
-    out.sel3 = sel3;
-    out.p13 = (addr1 ^ addr3p) & 0x2000u;  // r ^ q = p
-}
-
-// A flagged nibble (rank 4, stored as 8 | 2) makes PRMT return the sign fill of
-// pool entry 2 (c = 0: -1) or 6 (c = 1: 0) instead of the rank-4 value
-// (c = 0: -8, c = 1: 10).  Returns the coordinate inside the section, the
-// amount to add to y0 there, and the change of sum(y0^2).
-__device__ __forceinline__ void rank4_fix(uint32_t flags, uint32_t sel, int* j, int* dy, int* dsq) {
-    const int bit = __ffs(int(flags)) - 1;  // 4 j + 3
-    *j = bit >> 2;
-    const bool c = (sel >> (bit - 1)) & 1u;
-    *dy = c ? 10 : -7;    // 10 - 0, -8 - (-1)
-    *dsq = c ? 100 : 63;  // 100 - 0, 64 - 1
+    // p = r ^ q sits at bit 13 of both row addresses; 2^13 * 2^19 = 2^32 turns it into 0 / 1 on the
+    // multiplier pipe, and multiply-adds pick and patch the pools: the logic pipe sees one LOP3 of this
+    const uint32_t p = __umulhi((addr1 ^ addr3p) & 0x2000u, 0x80000u);
+    const uint32_t pool_lo = p * (kPool1Lo - kPool0Lo) + kPool0Lo;
+    const uint32_t pool_hi = p * (kPool1Hi - kPool0Hi) + kPool0Hi;
+    const uint32_t step = p * (2u * kRank4Step) - kRank4Step;  // (2p - 1) * (4 << 16)
+    const uint32_t f1 = top_slots_flag(w0 * 0x200000u);        // i1' in the top 11 bits
+    const uint32_t f3 = top_slots_flag(w0 * 0x200u);           // i3' in the top 11 bits
+    const uint32_t lo1 = f1 * step + pool_lo, hi1 = pool_hi - f1 * step;
+    const uint32_t lo3 = f3 * step + pool_lo, hi3 = pool_hi - f3 * step;
+    out.y[0] = prmt(lo1, hi1, sel1);
+    out.y[1] = prmt(lo1, hi1, sel1 >> 16);
+    out.y[2] = prmt(pool_lo, pool_hi, sel2);
+    out.y[3] = prmt(pool_lo, pool_hi, sel2 >> 16);
+    out.y[4] = prmt(lo3, hi3, sel3);
+    out.y[5] = prmt(lo3, hi3, sel3 >> 16);
 }
 
 }  // namespace tetra

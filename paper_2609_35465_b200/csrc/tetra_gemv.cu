@@ -164,7 +164,7 @@ struct LaneX {
     uint32_t mid[6];  // bits 15..8 (unsigned)
     uint32_t lo[6];   // bits 7..0 (unsigned)
     float step;       // 2^(E-22)
-    int sum;          // sum of q over the 24 coordinates
+    int sum;          // sum of q over the 24 coordinates (kept in the record; unused by the kernels)
 };
 
 __device__ __forceinline__ void lane_x_from_words(const uint32_t q[20], bool active, LaneX& X) {
@@ -178,67 +178,39 @@ __device__ __forceinline__ void lane_x_from_words(const uint32_t q[20], bool act
     X.sum = active ? int(q[19]) : 0;
 }
 
-// q of one coordinate, read back from a column's record (fix-up path only; the
-// record may sit in shared or in global memory).
-__device__ __forceinline__ int xq_coord(const unsigned char* rec, int coord) {
-    const int h = reinterpret_cast<const signed char*>(rec)[kXqHi + coord];
-    return h * 65536 + (int(rec[kXqMid + coord]) << 8 | int(rec[kXqLo + coord]));
-}
-
 // One block: device word -> contribution scale_b * sum_j y_j x_j (Eq. (2) without
-// the row scale).  xq_rec: this column's fixed-point record.
+// the row scale).
 template <bool HI>
-__device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint32_t w1pair, const LaneX& X,
-                                             const unsigned char* xq_rec) {
+__device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint32_t w1pair, const LaneX& X) {
     FastBlock fb;
     fast_decode<HI>(sm_tab, w0, w1pair, fb);
-    int dh = 0, dm = 0, dl = 0, n2 = 0, n1 = 0;
+    int dh = 0, dm = 0, dl = 0, n2 = 0;
 #pragma unroll
     for (int k = 0; k < 6; ++k) {
-        dh = dp4a_ss(fb.y0[k], X.hi[k], dh);
-        dm = dp4a_su(fb.y0[k], X.mid[k], dm);
-        dl = dp4a_su(fb.y0[k], X.lo[k], dl);
-        n2 = dp4a_ss(fb.y0[k], fb.y0[k], n2);
-        n1 = dp4a_ss(fb.y0[k], 0x01010101u, n1);
+        dh = dp4a_ss(fb.y[k], X.hi[k], dh);
+        dm = dp4a_su(fb.y[k], X.mid[k], dm);
+        dl = dp4a_su(fb.y[k], X.lo[k], dl);
+        n2 = dp4a_ss(fb.y[k], fb.y[k], n2);
     }
     // |sum_j y_j q_j| <= sqrt(24 * 416) * 2^23 < 2^31: the block's dot product is an exact int32
     int dot = dh * 65536 + (dm * 256 + dl);
-    if ((fb.row1 | fb.row3) & kRank4Flags) {  // a coordinate of rank 4: about 1.6 % of uniform random words
-        if (fb.row1 & kRank4Flags) {
-            int j, dy, dsq;
-            rank4_fix(fb.row1 & kRank4Flags, fb.sel1, &j, &dy, &dsq);
-            dot += dy * xq_coord(xq_rec, j);
-            n2 += dsq;
-            n1 += dy;
-        }
-        if (fb.row3 & kRank4Flags) {
-            int j, dy, dsq;
-            rank4_fix(fb.row3 & kRank4Flags, fb.sel3, &j, &dy, &dsq);
-            dot += dy * xq_coord(xq_rec, 16 + j);
-            n2 += dsq;
-            n1 += dy;
-        }
-    }
-    if (fb.p13) {  // p = 1: y = 1 - y0
-        dot = X.sum - dot;
-        n2 = n2 - 2 * n1 + 24;
-    }
-    // n2 = 16 m; the scale table holds gain[g] / sqrt(16 m) at 128 g + 4 m
-    const float scale = lds32f(fb.goff + (uint32_t(n2) >> 2));
+    // n2 = 16 m; the scale table holds gain[g] / sqrt(16 m) at 128 g + 4 m.  The index is masked into
+    // the table, so the load stays aligned and in bounds whatever the inputs are.
+    const float scale = lds32f(fb.goff | ((uint32_t(n2) >> 2) & 0x7Cu));
     return float(dot) * (scale * X.step);
 }
 
 // The eight blocks of one 48-byte record (rows 8G..8G+7 of one column).
 __device__ __forceinline__ void record_values(uint32_t sm_tab, const uint4& a, const uint4& b, const uint4& h,
-                                              const LaneX& X, const unsigned char* xq_rec, float v[8]) {
-    v[0] = block_value<false>(sm_tab, a.x, h.x, X, xq_rec);
-    v[1] = block_value<true>(sm_tab, a.y, h.x, X, xq_rec);
-    v[2] = block_value<false>(sm_tab, a.z, h.y, X, xq_rec);
-    v[3] = block_value<true>(sm_tab, a.w, h.y, X, xq_rec);
-    v[4] = block_value<false>(sm_tab, b.x, h.z, X, xq_rec);
-    v[5] = block_value<true>(sm_tab, b.y, h.z, X, xq_rec);
-    v[6] = block_value<false>(sm_tab, b.z, h.w, X, xq_rec);
-    v[7] = block_value<true>(sm_tab, b.w, h.w, X, xq_rec);
+                                              const LaneX& X, float v[8]) {
+    v[0] = block_value<false>(sm_tab, a.x, h.x, X);
+    v[1] = block_value<true>(sm_tab, a.y, h.x, X);
+    v[2] = block_value<false>(sm_tab, a.z, h.y, X);
+    v[3] = block_value<true>(sm_tab, a.w, h.y, X);
+    v[4] = block_value<false>(sm_tab, b.x, h.z, X);
+    v[5] = block_value<true>(sm_tab, b.y, h.z, X);
+    v[6] = block_value<false>(sm_tab, b.z, h.w, X);
+    v[7] = block_value<true>(sm_tab, b.w, h.w, X);
 }
 
 // Sums v[r] over the 32 lanes for r = 0..7 through the warp's shared-memory
@@ -340,7 +312,7 @@ k_gemv_fast(const DeviceTables* __restrict__ tab, const Problem single, int batc
                             n0 = __ldg(rec); n1 = __ldg(rec + B); n2 = __ldg(rec + 2 * size_t(B));
                         }
                         float v[8];
-                        record_values(sm_tab, a, b, h, X, xq_rec, v);
+                        record_values(sm_tab, a, b, h, X, v);
                         float sum = transpose_partial(red, lane, v);
                         sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
                         sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
@@ -451,7 +423,13 @@ __global__ void __launch_bounds__(256) k_prepare_x(unsigned char* __restrict__ w
     }
 }
 
-__global__ void __launch_bounds__(kFastThreads, 1)
+#ifndef TETRA_UNIT_THREADS
+#define TETRA_UNIT_THREADS 512
+#endif
+constexpr int kUnitThreads = TETRA_UNIT_THREADS;
+constexpr int kUnitWarps = kUnitThreads / 32;
+
+__global__ void __launch_bounds__(kUnitThreads, 1)
 k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restrict__ ws) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     unsigned char* smem = stage_fast_tables(tab, smem_raw);
@@ -467,7 +445,7 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
     const unsigned char* xq_all = ws + H->off_xq;
     const int count = H->count, total_units = H->total_units;
     // consecutive units (neighbouring row groups of a matrix) go to consecutive warps of the grid
-    for (int u = blockIdx.x * kFastWarps + warp; u < total_units; u += gridDim.x * kFastWarps) {
+    for (int u = blockIdx.x * kUnitWarps + warp; u < total_units; u += gridDim.x * kUnitWarps) {
         const int p = find_problem(unit_prefix, count, u);
         const int g = u - __ldg(unit_prefix + p);
         const Problem P = problems[p];
@@ -504,7 +482,7 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
                 X.sum = int(t4.w);
             }
             float v[8];
-            record_values(sm_tab, a, b, h, X, xq_rec, v);
+            record_values(sm_tab, a, b, h, X, v);
 #pragma unroll
             for (int r = 0; r < 8; ++r) acc[r] += v[r];
         }
@@ -586,7 +564,7 @@ cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s) {
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
-    const uint32_t smem = kTableSmemBytes + kFastWarps * kRedFloats * 4;
+    const uint32_t smem = kTableSmemBytes + kUnitWarps * kRedFloats * 4;
     if (!attr_set[dev]) {
         e = cudaFuncSetAttribute(k_gemv_units, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
         if (e != cudaSuccess) return e;
@@ -595,7 +573,7 @@ cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s) {
     k_prepare_x<<<sms * 2, 256, 0, s>>>(static_cast<unsigned char*>(ws_dev));
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    k_gemv_units<<<sms, kFastThreads, smem, s>>>(static_cast<const DeviceTables*>(table),
+    k_gemv_units<<<sms, kUnitThreads, smem, s>>>(static_cast<const DeviceTables*>(table),
                                                  static_cast<const unsigned char*>(ws_dev));
     return cudaGetLastError();
 }

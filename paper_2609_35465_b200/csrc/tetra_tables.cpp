@@ -170,23 +170,62 @@ int build_device_tables(DeviceTables* out, const float* gain2) {
     out->magic = kTableMagic;
     out->version = kTableVersion;
 
-    // Fast-path rows: ranks 0..3 stay; rank 4 becomes 8 | 2.
-    for (int i = 0; i < 4096; ++i) {
-        uint32_t row = out->paper.rows[i], fast = 0;
-        int flagged = 0;
-        for (int j = 0; j < 8; ++j) {
-            unsigned r = (row >> (4 * j)) & 15u;
-            if (r > 4) return -21;
-            if (r == 4) { r = 8u | 2u; ++flagged; }
-            fast |= r << (4 * j);
+    // Fast-path rows.  Per class: rows holding a rank-4 coordinate go to the last
+    // kRank4Slots slots, topped up with rows that use ranks 0 and 1 only (a patched
+    // pool serves ranks 0, 1 and 4); everything else keeps its order in front.
+    for (int cls = 0; cls < 2; ++cls) {
+        std::vector<int> tail_rows, fillers, front;
+        for (int i = 0; i < 2048; ++i) {
+            const uint32_t row = out->paper.rows[2048 * cls + i];
+            int max_rank = 0, n4 = 0;
+            for (int j = 0; j < 8; ++j) {
+                const int r = (row >> (4 * j)) & 15;
+                if (r > 4) return -21;
+                if (r == 4) ++n4;
+                if (r > max_rank) max_rank = r;
+            }
+            if (n4 > 1) return -22;
+            if (n4 == 1) {
+                for (int j = 0; j < 8; ++j) {  // the other coordinates of such a row are of rank 0 or 1
+                    const int r = (row >> (4 * j)) & 15;
+                    if (r == 2 || r == 3) return -24;
+                }
+                tail_rows.push_back(i);
+            } else if (max_rank <= 1) {
+                fillers.push_back(i);
+            } else {
+                front.push_back(i);
+            }
         }
-        if (flagged > 1) return -22;  // the fix-up path handles one coordinate per section
-        out->rows_fast[i] = fast;
+        if (int(tail_rows.size()) > kRank4Slots) return -25;
+        while (int(tail_rows.size()) < kRank4Slots) {
+            if (fillers.empty()) return -26;
+            tail_rows.push_back(fillers.back());
+            fillers.pop_back();
+        }
+        front.insert(front.end(), fillers.begin(), fillers.end());
+        std::sort(front.begin(), front.end());
+        if (int(front.size()) != 2048 - kRank4Slots) return -27;
+        for (int slot = 0; slot < 2048; ++slot) {
+            const int i = slot < int(front.size()) ? front[slot] : tail_rows[slot - int(front.size())];
+            const uint32_t row = out->paper.rows[2048 * cls + i];
+            uint32_t fast = 0;
+            for (int j = 0; j < 8; ++j) {
+                unsigned r = (row >> (4 * j)) & 15u;
+                if (r == 4) r = 2;
+                fast |= r << (4 * j);
+            }
+            out->rows_fast[2048 * cls + slot] = fast;
+            out->row_perm[cls][i] = static_cast<uint16_t>(slot);
+        }
     }
+    // The middle list keeps its own copy in i2 order; its rows never reach rank 4.
     for (int i2 = 0; i2 < 2048; ++i2) {
         const int idx = i2 < n0 ? i2 : 2048 + (i2 - n0);
-        if (out->rows_fast[idx] & 0x88888888u) return -23;  // middle rows never reach rank 4
-        out->mid_fast[i2] = out->rows_fast[idx];
+        const uint32_t row = out->paper.rows[idx];
+        for (int j = 0; j < 8; ++j)
+            if (((row >> (4 * j)) & 15u) > 3) return -23;
+        out->mid_fast[i2] = row;
     }
     for (unsigned v = 0; v < 16; ++v) {
         const uint8_t h = span4(turyn.h, v), hr = span4(turyn.hr, v);

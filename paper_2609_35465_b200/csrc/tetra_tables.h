@@ -17,7 +17,8 @@ struct PaperTables {
 static_assert(sizeof(PaperTables) == 18816, "paper table blob is 18,816 bytes");
 
 constexpr uint32_t kTableMagic = 0x54455442u;  // "TETB"
-constexpr uint32_t kTableVersion = 4;
+constexpr uint32_t kTableVersion = 5;
+constexpr int kRank4Slots = 32;                // slots at the end of each class whose pool is patched
 constexpr int kMiddleClass0 = 1240;            // N0 of Sec. 3.3 (checked at build)
 
 // Everything tetra_build_table copies to the device, in one blob.
@@ -27,8 +28,11 @@ struct DeviceTables {
     uint32_t magic;             // 18824
     uint32_t version;           // 18828
     // ---- fast path: everything below is staged in shared memory ------------
-    // Rank rows for PRMT lookup: nibble j = rank (0..3); a coordinate of rank 4
-    // is stored as 8 | 2 (bit 3 flags it for the fix-up path).
+    // Rank rows for PRMT lookup, class by class in the permuted order of
+    // row_perm: nibble j = rank (0..3).  The last 32 slots of each class hold the
+    // rows with a coordinate of rank 4 (stored there as rank 2) and, as fillers,
+    // rows that use ranks 0 and 1 only: for those slots the kernels patch the
+    // rank-2 entries of the PRMT pool to the rank-4 values.
     // (the kernels place this part on a 16 KiB boundary of shared memory, so each
     //  sub-table's offset can be OR-ed into an index instead of added)
     uint32_t rows_fast[4096];   // +0
@@ -42,6 +46,8 @@ struct DeviceTables {
     // ---- pack-time only (global memory) ------------------------------------
     // 12 trellis bits (s8 | b1<<6 | b2<<7 | b3<<11) -> Turyn coordinates a | b<<4 | x<<8.
     uint16_t trellis_to_abx[4096];
+    // row_perm[cls][i]: slot of file-order row 2048 cls + i inside its class of rows_fast.
+    uint16_t row_perm[2][2048];
 };
 
 constexpr size_t kFastOffset = offsetof(DeviceTables, rows_fast);

@@ -11,7 +11,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libtetra_b200.so")
+LIB_PATH = os.environ.get("TETRA_LIB") or os.path.join(_HERE, "libtetra_b200.so")
 
 BLOCK = 24
 WORD_BYTES = 6
