@@ -29,10 +29,11 @@ METRIC = "tetra_gemv_batch1_hbm_gbps"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per algorithmic byte of the grouped kernel, from the ncu capture
-# summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on one
-# Qwen3-8B layer, 49 MB of codes; traffic grows in proportion to the matrices read).
-TRAFFIC_PER_ALGORITHMIC_BYTE = None
+# DRAM bytes per algorithmic byte of k_gemv_units, from the ncu capture summarised in
+# profiles/k_gemv_units_qwen3_8b.md (dram__bytes_read.sum + dram__bytes_write.sum = 202.5 MB
+# for the 198.4 MB of the first 4 layers; every code byte is read once, so traffic grows in
+# proportion to the matrices read and the full pass is scaled by its byte count).
+TRAFFIC_PER_ALGORITHMIC_BYTE = 1.02
 
 
 def measured_peak():
@@ -185,7 +186,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2609_35465_b200 import shapes
+    from paper_2609_35465_b200 import ranks, shapes
     from paper_2609_35465_b200 import build as tbuild
     from paper_2609_35465_b200.workload import DevicePass
 
@@ -227,20 +228,12 @@ def main():
     e1.record(stream)
     barrier()
     clocks = sampler.stop()
-    ms = e0.elapsed_time(e1) / args.steps
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = ranks.max_over_ranks(e0.elapsed_time(e1) / args.steps, device="cuda")
     y_grouped = dp.y_all.cpu().numpy().copy()
 
     # ---- end to end: activations from pinned host memory, results back to it
     e2e_steps = max(3, min(args.steps, 200))
-    e2e_ms = timed(torch, dp.run_grouped_hostio, e2e_steps, 3, stream)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = ranks.max_over_ranks(timed(torch, dp.run_grouped_hostio, e2e_steps, 3, stream), device="cuda")
     assert np.array_equal(dp.y_host.numpy(), y_grouped), "host-io result differs from the device-resident run"
 
     if rank != 0:
@@ -274,7 +267,7 @@ def main():
                 "d2h_bytes_per_step": int(dp.y_host.numel() * 4),
                 "api": "tetra_gemv_grouped_hostio: activations from pinned host memory, results to it; "
                        "codes, scales and tails stay resident in HBM as model weights do"},
-        "roofline": {"bound": "hbm", "kernel": "k_gemv_fast", "achieved": gbs, "peak": peak, "unit": "GB/s",
+        "roofline": {"bound": "hbm", "kernel": "k_gemv_units", "achieved": gbs, "peak": peak, "unit": "GB/s",
                      "frac": gbs / peak, "peak_kind": peak_kind + " copy bandwidth",
                      "traffic": (None if TRAFFIC_PER_ALGORITHMIC_BYTE is None
                                  else TRAFFIC_PER_ALGORITHMIC_BYTE * dp.algorithmic_bytes),

@@ -1,0 +1,96 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py
+times (a planned list run by tetra_gemv_grouped_run), on sampled output rows
+the oracle computes one by one; plus properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_35465_b200 import shapes, synth
+from helpers import assert_gemv_close, oracle_product
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_sampled(dp, orc, picks, rows_per_matrix=6, seed=0):
+    rng = np.random.default_rng(seed)
+    y_all = dp.y_all.cpu().numpy()
+    worst = 0.0
+    for i in picks:
+        it = dp.items[i]
+        rows = np.unique(np.concatenate([[0, it["N"] - 1], rng.integers(0, it["N"], rows_per_matrix)]))
+        m = dp.host_inputs(i, rows=rows)
+        ref = oracle_product(orc, m, dp.gain, threads=1)
+        y = y_all[it["yoff"]:it["yoff"] + it["N"]][rows]
+        _, w = assert_gemv_close(y, ref, it["name"])
+        worst = max(worst, w)
+    return worst
+
+
+def test_qwen3_8b_full_pass_sampled_rows(orc):
+    """Config 2: all 252 matrices of the Qwen3-8B-shaped pass in one planned run."""
+    from paper_2609_35465_b200.workload import DevicePass
+    dp = DevicePass(shapes.QWEN3_8B.all_matrices(), seed=0)
+    dp.y_all.fill_(float("nan"))
+    dp.run_grouped()
+    torch.cuda.synchronize()
+    y = dp.y_all.cpu().numpy()
+    used = np.zeros(len(y), dtype=bool)
+    for it in dp.items:
+        used[it["yoff"]:it["yoff"] + it["N"]] = True
+    assert np.isfinite(y[used]).all()                     # every output row was written
+    assert dp.algorithmic_bytes == 1785397248
+    picks = list(range(7)) + [7 * 17 + k for k in range(7)] + list(range(245, 252))
+    _check_sampled(dp, orc, picks)
+    # rerun: bit-identical (fixed summation order, no atomics)
+    dp.run_grouped()
+    torch.cuda.synchronize()
+    assert np.array_equal(dp.y_all.cpu().numpy()[used], y[used])
+    # the host-buffer entry point gives the same bits
+    dp.y_all.zero_()
+    dp.run_grouped_hostio()
+    torch.cuda.synchronize()
+    assert np.array_equal(dp.y_host.numpy()[used], y[used])
+
+
+def test_qwen3_14b_layers_sampled_rows(orc):
+    """Config 3 shapes (hidden 5120, intermediate 17408: 213 and 725 words per row, tails of 8)."""
+    from paper_2609_35465_b200.workload import DevicePass
+    mats = shapes.QWEN3_14B.all_matrices()[:14]
+    dp = DevicePass(mats, seed=3)
+    dp.run_grouped()
+    torch.cuda.synchronize()
+    _check_sampled(dp, orc, range(len(mats)), rows_per_matrix=4, seed=3)
+
+
+def test_qwen3_4b_layer_zero_pad_rule(orc):
+    """Config 1 with K zero-padded to a multiple of 24 instead of the tail rule."""
+    from paper_2609_35465_b200.workload import DevicePass
+    mats = shapes.QWEN3_4B.layer_matrices()
+    dp = DevicePass(mats, seed=4, tail_mode=False)
+    assert all(it["ntail"] == 0 and it["B"] == -(-it["K"] // 24) for it in dp.items)
+    dp.run_grouped()
+    torch.cuda.synchronize()
+    _check_sampled(dp, orc, range(len(mats)), rows_per_matrix=8, seed=4)
+
+
+@pytest.mark.parametrize("batch", shapes.CONFIG4_BATCHES)
+def test_down_proj_batch_sweep_sampled_rows(orc, batch):
+    """Config 4: N = 4096, K = 12288 with 1..16 activation vectors."""
+    from paper_2609_35465_b200 import tetra as tt
+    m = shapes.CONFIG4
+    table = tt.tetra_build_table(synth.DEFAULT_GAIN)
+    codes = synth.codes_torch(6, 1, m.N, m.blocks, device="cuda")
+    packed = tt.tetra_pack_codes(codes, table, m.N, m.blocks)
+    sigma = synth.row_scales(6, 1, m.N)
+    x = synth.activations(6, 1, m.K, batch)
+    y = torch.full((batch, m.N), float("nan"), dtype=torch.float32, device="cuda")
+    tt.tetra_gemv(packed, torch.from_numpy(sigma).cuda(), table, torch.from_numpy(x).cuda(), y, m.N, m.K, batch)
+    torch.cuda.synchronize()
+    yh = y.cpu().numpy()
+    assert np.isfinite(yh).all()
+    rows = np.array([0, 1, 2047, 4095, 1234, 3001])
+    host_codes = np.stack([synth.words_to_bytes(synth.words(6, 1, m.blocks, int(r) * m.blocks)) for r in rows])
+    for b in sorted({0, batch - 1}):
+        mm = dict(N=len(rows), K=m.K, B=m.blocks, ntail=0, codes=host_codes, sigma=sigma[rows], x=x, tail=None)
+        ref = oracle_product(orc, mm, synth.DEFAULT_GAIN, batch_index=b, threads=1)
+        assert_gemv_close(yh[b][rows], ref, "batch %d column %d" % (batch, b))
