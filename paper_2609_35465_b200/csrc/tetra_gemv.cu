@@ -374,17 +374,22 @@ cudaError_t launch_gemv_fast(const Problem& single, int batch, int max_blocks, c
 // Planned list of matrices: k_prepare_x + k_gemv_units
 // ===========================================================================
 // Workspace written by grouped_plan (host) and read by both kernels:
-//   PlanHeader | Problem[count] | unit_prefix[count + 1] | col_prefix[count + 1] | pad | xq records
+//   PlanHeader | Problem[count] | unit_prefix[count + 1] | col_prefix[count + 1]
+//              | warp_start[nwarps + 1] (optional) | pad | xq records
 struct PlanHeader {
     int32_t count;
     int32_t total_units;  // sum over matrices of ceil(N / 8)
     int32_t total_cols;   // sum over matrices of words per row
-    int32_t reserved;
+    int32_t nwarps;       // warps the unit ranges were cut for (0: no ranges, units are dealt round-robin)
     uint32_t off_problems, off_unit_prefix, off_col_prefix, off_xq;
+    uint32_t off_warp_start, pad_[3];
 };
 
-static size_t plan_meta_bytes(int count) {
-    size_t b = sizeof(PlanHeader) + size_t(count) * sizeof(Problem) + 2 * size_t(count + 1) * 4;
+constexpr int kMaxPlanWarps = 8192;  // room reserved for warp_start in a planned list's workspace
+
+static size_t plan_meta_bytes(int count, int nwarps) {
+    size_t b = sizeof(PlanHeader) + size_t(count) * sizeof(Problem) + 2 * size_t(count + 1) * 4 +
+               (nwarps ? size_t(nwarps + 1) * 4 : 0);
     return (b + 255) & ~size_t(255);
 }
 
@@ -395,7 +400,7 @@ static inline int problem_blocks(const Problem& q) {
 size_t grouped_workspace_bytes(const Problem* problems, int count) {
     size_t cols = 0;
     for (int i = 0; i < count; ++i) cols += size_t(problem_blocks(problems[i]));
-    return plan_meta_bytes(count) + cols * kXqBytesPerCol;
+    return plan_meta_bytes(count, kMaxPlanWarps) + cols * kXqBytesPerCol;
 }
 
 // Largest p with prefix[p] <= v (prefix[0] = 0, prefix[count] > v).
@@ -443,32 +448,66 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
     const int32_t* unit_prefix = reinterpret_cast<const int32_t*>(ws + H->off_unit_prefix);
     const int32_t* col_prefix = reinterpret_cast<const int32_t*>(ws + H->off_col_prefix);
     const unsigned char* xq_all = ws + H->off_xq;
-    const int count = H->count, total_units = H->total_units;
-    // consecutive units (neighbouring row groups of a matrix) go to consecutive warps of the grid
-    for (int u = blockIdx.x * kUnitWarps + warp; u < total_units; u += gridDim.x * kUnitWarps) {
-        const int p = find_problem(unit_prefix, count, u);
-        const int g = u - __ldg(unit_prefix + p);
-        const Problem P = problems[p];
-        const int ntail = P.tail ? P.K % 24 : 0;
-        const int B = P.tail ? P.K / 24 : (P.K + 23) / 24;
-        const int CG = (B + 31) / 32;
-        const unsigned char* xq_p = xq_all + size_t(__ldg(col_prefix + p)) * kXqBytesPerCol;
-        const uint4* codes = static_cast<const uint4*>(P.codes) + size_t(g) * 3 * B;
+    const int total_units = H->total_units;
+
+    // Units of this warp: a contiguous range cut for equal work when the plan holds ranges for this
+    // grid (neighbouring warps then walk neighbouring row groups of the same matrices), else every
+    // (warps in grid)-th unit.
+    const int gw = blockIdx.x * kUnitWarps + warp, nw = gridDim.x * kUnitWarps;
+    int u = gw, u_end = total_units, u_step = nw;
+    if (H->nwarps == nw) {
+        const int32_t* warp_start = reinterpret_cast<const int32_t*>(ws + H->off_warp_start);
+        u = __ldg(warp_start + gw);
+        u_end = __ldg(warp_start + gw + 1);
+        u_step = 1;
+    }
+    int p = -1, p_begin = 0, p_end = 0;  // matrix of the current unit and its range of units
+    Problem P{};
+    int ntail = 0, B = 1, CG = 1;
+    const unsigned char* xq_p = xq_all;
+    bool have_record = false;  // n0..n2 already hold the first record of the unit about to start
+    uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0, n2 = n0;
+
+    for (; u < u_end; u += u_step) {
+        if (u >= p_end) {  // first unit, or the walk has left the matrix: units only go up
+            do { ++p; p_end = __ldg(unit_prefix + p + 1); } while (u >= p_end);
+            p_begin = __ldg(unit_prefix + p);
+            P = problems[p];
+            ntail = P.tail ? P.K % 24 : 0;
+            B = P.tail ? P.K / 24 : (P.K + 23) / 24;
+            CG = (B + 31) / 32;
+            xq_p = xq_all + size_t(__ldg(col_prefix + p)) * kXqBytesPerCol;
+            have_record = false;
+        }
+        const int g = u - p_begin;
+        const uint32_t Bu = uint32_t(B);
+        const uint4* codes = static_cast<const uint4*>(P.codes) + size_t(g) * 3 * Bu;
 
         float acc[8];
 #pragma unroll
         for (int r = 0; r < 8; ++r) acc[r] = 0.f;
         // lanes beyond the last column re-read column B - 1 and contribute with a zero step
-        const uint32_t Bu = uint32_t(B);
         uint32_t col = min(uint32_t(lane), Bu - 1);
-        uint4 n0 = __ldg(codes + col), n1 = __ldg(codes + Bu + col), n2 = __ldg(codes + 2 * Bu + col);
+        if (!have_record) {
+            n0 = __ldg(codes + col); n1 = __ldg(codes + Bu + col); n2 = __ldg(codes + 2 * Bu + col);
+        }
         for (int cg = 0; cg < CG; ++cg) {
             const bool active = uint32_t(cg * 32 + lane) < Bu;
             const uint4 a = n0, b = n1, h = n2;
             const unsigned char* xq_rec = xq_p + col * uint32_t(kXqBytesPerCol);
-            col = min(uint32_t((cg + 1) * 32 + lane), Bu - 1);
-            if (cg + 1 < CG) {  // prefetch the next column group's record
-                n0 = __ldg(codes + col); n1 = __ldg(codes + Bu + col); n2 = __ldg(codes + 2 * Bu + col);
+            // prefetch the next record: the next column group, or the first one of this warp's next unit
+            have_record = false;
+            const uint4* next = codes;
+            if (cg + 1 < CG) {
+                col = min(uint32_t((cg + 1) * 32 + lane), Bu - 1);
+                have_record = true;
+            } else if (u + u_step < min(u_end, p_end)) {
+                col = min(uint32_t(lane), Bu - 1);
+                next = codes + size_t(u_step) * 3 * Bu;
+                have_record = true;
+            }
+            if (have_record) {
+                n0 = __ldg(next + col); n1 = __ldg(next + Bu + col); n2 = __ldg(next + 2 * Bu + col);
             }
             LaneX X;
             {
@@ -502,16 +541,23 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
 }
 
 cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, size_t ws_bytes, cudaStream_t s) {
-    const size_t meta = plan_meta_bytes(count);
     if (ws_bytes < grouped_workspace_bytes(problems_host, count)) return cudaErrorInvalidValue;
+    int sms = 0;
+    cudaError_t e = device_sms(&sms);
+    if (e != cudaSuccess) return e;
+    int nwarps = sms * kUnitWarps;  // the grid grouped_run launches on this device
+    if (nwarps > kMaxPlanWarps) nwarps = 0;
+    const size_t meta = plan_meta_bytes(count, nwarps);
     unsigned char* buf = static_cast<unsigned char*>(calloc(1, meta));
     if (!buf) return cudaErrorMemoryAllocation;
     PlanHeader* H = reinterpret_cast<PlanHeader*>(buf);
     H->count = count;
+    H->nwarps = nwarps;
     H->off_problems = uint32_t(sizeof(PlanHeader));
     H->off_unit_prefix = H->off_problems + uint32_t(count) * uint32_t(sizeof(Problem));
     H->off_col_prefix = H->off_unit_prefix + uint32_t(count + 1) * 4u;
-    H->off_xq = uint32_t(meta);
+    H->off_warp_start = H->off_col_prefix + uint32_t(count + 1) * 4u;
+    H->off_xq = uint32_t(plan_meta_bytes(count, kMaxPlanWarps));
     memcpy(buf + H->off_problems, problems_host, size_t(count) * sizeof(Problem));
     int32_t* up = reinterpret_cast<int32_t*>(buf + H->off_unit_prefix);
     int32_t* cp = reinterpret_cast<int32_t*>(buf + H->off_col_prefix);
@@ -524,32 +570,53 @@ cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, 
     }
     up[count] = int32_t(units);
     cp[count] = int32_t(cols);
-    cudaError_t e = cudaSuccess;
     if (units > 0x7FFFFFF0LL || cols > 0x7FFFFFF0LL) e = cudaErrorInvalidValue;
     H->total_units = int32_t(units);
     H->total_cols = int32_t(cols);
+    if (e == cudaSuccess && nwarps) {
+        // Cut the unit sequence into nwarps contiguous ranges of equal work; a unit costs its number of
+        // column groups plus a little for its prologue and epilogue.
+        auto unit_work = [&](int i) { return (long long)((problem_blocks(problems_host[i]) + 31) / 32) * 8 + 2; };
+        long long total = 0;
+        for (int i = 0; i < count; ++i) total += unit_work(i) * ((problems_host[i].N + 7) / 8);
+        int32_t* wsx = reinterpret_cast<int32_t*>(buf + H->off_warp_start);
+        int pi = 0;
+        long long before = 0;  // work of matrices 0..pi-1
+        for (int w = 0; w < nwarps; ++w) {
+            const long long target = total * w / nwarps;
+            while (pi < count - 1 && before + unit_work(pi) * ((problems_host[pi].N + 7) / 8) <= target) {
+                before += unit_work(pi) * ((problems_host[pi].N + 7) / 8);
+                ++pi;
+            }
+            long long uu = up[pi] + (target - before) / unit_work(pi);
+            if (uu > units) uu = units;
+            wsx[w] = int32_t(uu);
+        }
+        wsx[nwarps] = int32_t(units);
+    }
     // pageable source: the runtime stages it before returning, so the buffer can be freed
     if (e == cudaSuccess) e = cudaMemcpyAsync(ws_dev, buf, meta, cudaMemcpyHostToDevice, s);
     free(buf);
     return e;
 }
 
-size_t single_plan_meta_bytes() { return plan_meta_bytes(1); }
+size_t single_plan_meta_bytes() { return plan_meta_bytes(1, 0); }
 
 size_t single_plan_scratch_bytes(int blocks_per_row) {
-    return plan_meta_bytes(1) + size_t(blocks_per_row) * kXqBytesPerCol;
+    return plan_meta_bytes(1, 0) + size_t(blocks_per_row) * kXqBytesPerCol;
 }
 
 void single_plan_fill(const Problem& problem, unsigned char* meta_host) {
-    memset(meta_host, 0, plan_meta_bytes(1));
+    memset(meta_host, 0, plan_meta_bytes(1, 0));
     PlanHeader* H = reinterpret_cast<PlanHeader*>(meta_host);
     H->count = 1;
     H->total_units = (problem.N + 7) / 8;
     H->total_cols = problem_blocks(problem);
     H->off_problems = uint32_t(sizeof(PlanHeader));
+    H->nwarps = 0;  // no unit ranges: the kernel deals units round-robin
     H->off_unit_prefix = H->off_problems + uint32_t(sizeof(Problem));
     H->off_col_prefix = H->off_unit_prefix + 8u;
-    H->off_xq = uint32_t(plan_meta_bytes(1));
+    H->off_xq = uint32_t(plan_meta_bytes(1, 0));
     memcpy(meta_host + H->off_problems, &problem, sizeof(Problem));
     int32_t* up = reinterpret_cast<int32_t*>(meta_host + H->off_unit_prefix);
     int32_t* cp = reinterpret_cast<int32_t*>(meta_host + H->off_col_prefix);
