@@ -376,9 +376,10 @@ cudaError_t launch_gemv_fast(const Problem& single, int batch, int max_blocks, c
 // Workspace written by grouped_plan (host) and read by both kernels:
 //   PlanHeader | Problem[count] | unit_prefix[count + 1] | col_prefix[count + 1]
 //              | warp_start[nwarps + 1] (optional) | pad | xq records
+// A unit is groups_per_unit(B) consecutive row groups of one matrix, all columns.
 struct PlanHeader {
     int32_t count;
-    int32_t total_units;  // sum over matrices of ceil(N / 8)
+    int32_t total_units;  // sum over matrices of their units
     int32_t total_cols;   // sum over matrices of words per row
     int32_t nwarps;       // warps the unit ranges were cut for (0: no ranges, units are dealt round-robin)
     uint32_t off_problems, off_unit_prefix, off_col_prefix, off_xq;
@@ -395,6 +396,20 @@ static size_t plan_meta_bytes(int count, int nwarps) {
 
 static inline int problem_blocks(const Problem& q) {
     return (q.tail || q.K % 24 == 0) ? q.K / 24 : (q.K + 23) / 24;
+}
+
+// Row groups (of eight rows) one unit covers.  When the last column group of a matrix is at most
+// half full (B mod 32 in 1..16), up to three consecutive row groups share one pass over it, so that
+// pass runs with most lanes busy instead of B mod 32 of them.
+__host__ __device__ inline int groups_per_unit(int B) {
+    const int rem = B & 31;
+    if (rem == 0 || rem > 16) return 1;
+    const int r = 32 / rem;
+    return r < 3 ? r : 3;
+}
+static inline int problem_units(const Problem& q) {
+    const int R = groups_per_unit(problem_blocks(q));
+    return ((q.N + 7) / 8 + R - 1) / R;
 }
 
 size_t grouped_workspace_bytes(const Problem* problems, int count) {
@@ -426,6 +441,17 @@ __global__ void __launch_bounds__(256) k_prepare_x(unsigned char* __restrict__ w
 #pragma unroll
         for (int k = 0; k < 5; ++k) xq[size_t(gc) * 5 + k] = make_uint4(q[4 * k], q[4 * k + 1], q[4 * k + 2], q[4 * k + 3]);
     }
+}
+
+// This lane's activation record (global memory, L1/L2 resident) into registers.
+__device__ __forceinline__ void load_lane_x(const unsigned char* xq_rec, bool active, LaneX& X) {
+    const uint4* src = reinterpret_cast<const uint4*>(xq_rec);
+    const uint4 t0 = __ldg(src), t1 = __ldg(src + 1), t2 = __ldg(src + 2), t3 = __ldg(src + 3), t4 = __ldg(src + 4);
+    X.hi[0] = t0.x; X.hi[1] = t0.y; X.hi[2] = t0.z; X.hi[3] = t0.w; X.hi[4] = t1.x; X.hi[5] = t1.y;
+    X.mid[0] = t1.z; X.mid[1] = t1.w; X.mid[2] = t2.x; X.mid[3] = t2.y; X.mid[4] = t2.z; X.mid[5] = t2.w;
+    X.lo[0] = t3.x; X.lo[1] = t3.y; X.lo[2] = t3.z; X.lo[3] = t3.w; X.lo[4] = t4.x; X.lo[5] = t4.y;
+    X.step = active ? __uint_as_float(t4.z) : 0.f;  // an inactive lane contributes exact zeros
+    X.sum = int(t4.w);
 }
 
 #ifndef TETRA_UNIT_THREADS
@@ -462,81 +488,118 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
         u_step = 1;
     }
     int p = -1, p_begin = 0, p_end = 0;  // matrix of the current unit and its range of units
-    Problem P{};
-    int ntail = 0, B = 1, CG = 1;
+    // per matrix, kept in registers across its units (everything else is re-read where it is needed)
+    const uint4* codes_p = nullptr;
     const unsigned char* xq_p = xq_all;
-    bool have_record = false;  // n0..n2 already hold the first record of the unit about to start
+    int G = 1;
+    uint32_t Bu = 1;
+    bool have_record = false;            // n0..n2 already hold the first record of the unit about to start
     uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0, n2 = n0;
 
     for (; u < u_end; u += u_step) {
         if (u >= p_end) {  // first unit, or the walk has left the matrix: units only go up
             do { ++p; p_end = __ldg(unit_prefix + p + 1); } while (u >= p_end);
             p_begin = __ldg(unit_prefix + p);
-            P = problems[p];
-            ntail = P.tail ? P.K % 24 : 0;
-            B = P.tail ? P.K / 24 : (P.K + 23) / 24;
-            CG = (B + 31) / 32;
+            const Problem& Q = problems[p];
+            const int K = Q.K;
+            Bu = uint32_t(Q.tail ? K / 24 : (K + 23) / 24);
+            G = (Q.N + 7) / 8;
+            codes_p = static_cast<const uint4*>(Q.codes);
             xq_p = xq_all + size_t(__ldg(col_prefix + p)) * kXqBytesPerCol;
             have_record = false;
         }
-        const int g = u - p_begin;
-        const uint32_t Bu = uint32_t(B);
-        const uint4* codes = static_cast<const uint4*>(P.codes) + size_t(g) * 3 * Bu;
+        const int CGf = int(Bu >> 5);   // full column groups
+        const int rem = int(Bu & 31);   // columns of the last, partial one
+        const int R = groups_per_unit(int(Bu));
+        const int g0 = (u - p_begin) * R;
+        const int ng = min(R, G - g0);
+        const uint4* codes0 = codes_p + size_t(g0) * 3 * Bu;
+        // this lane's place in the joint pass over the partial column group: row group, column
+        const int lane_grp = rem ? min(lane / max(rem, 1), 3) : 0;
+        const bool lane_in = rem && lane_grp < ng;
+        const uint32_t lane_col = uint32_t(CGf * 32) + (lane_in ? uint32_t(lane - lane_grp * rem) : 0u);
+        const uint4* rem_rec = codes0 + size_t(lane_in ? lane_grp : 0) * 3 * Bu + lane_col;
+        const bool next_unit_here = CGf > 0 && u + u_step < min(u_end, p_end);
 
+        if (!have_record) {
+            const uint4* first = CGf > 0 ? codes0 + lane : rem_rec;
+            n0 = __ldg(first); n1 = __ldg(first + Bu); n2 = __ldg(first + 2 * Bu);
+        }
+        have_record = false;
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f;  // per row group: this lane's partial row sum (row lane / 4)
         float acc[8];
 #pragma unroll
         for (int r = 0; r < 8; ++r) acc[r] = 0.f;
-        // lanes beyond the last column re-read column B - 1 and contribute with a zero step
-        uint32_t col = min(uint32_t(lane), Bu - 1);
-        if (!have_record) {
-            n0 = __ldg(codes + col); n1 = __ldg(codes + Bu + col); n2 = __ldg(codes + 2 * Bu + col);
-        }
-        for (int cg = 0; cg < CG; ++cg) {
-            const bool active = uint32_t(cg * 32 + lane) < Bu;
+
+        // One pass = one 48-byte record per lane: the full column groups of each row group in turn,
+        // then the joint pass over the partial column group (a single call site of the decoder).
+        const int full_passes = ng * CGf, passes = full_passes + (rem ? 1 : 0);
+        int gi = 0, cg = 0;
+        for (int pass = 0; pass < passes; ++pass) {
+            const bool joint = pass >= full_passes;
             const uint4 a = n0, b = n1, h = n2;
-            const unsigned char* xq_rec = xq_p + col * uint32_t(kXqBytesPerCol);
-            // prefetch the next record: the next column group, or the first one of this warp's next unit
-            have_record = false;
-            const uint4* next = codes;
-            if (cg + 1 < CG) {
-                col = min(uint32_t((cg + 1) * 32 + lane), Bu - 1);
-                have_record = true;
-            } else if (u + u_step < min(u_end, p_end)) {
-                col = min(uint32_t(lane), Bu - 1);
-                next = codes + size_t(u_step) * 3 * Bu;
+            // prefetch the next pass's record (or the first one of this warp's next unit)
+            const uint4* next = nullptr;
+            if (pass + 1 < full_passes) {
+                const bool wrap = cg + 1 == CGf;
+                next = codes0 + size_t(wrap ? gi + 1 : gi) * 3 * Bu + (wrap ? 0 : cg + 1) * 32 + lane;
+            } else if (pass + 1 < passes) {
+                next = rem_rec;
+            } else if (next_unit_here) {
+                next = codes0 + size_t(u_step) * R * 3 * Bu + lane;
                 have_record = true;
             }
-            if (have_record) {
-                n0 = __ldg(next + col); n1 = __ldg(next + Bu + col); n2 = __ldg(next + 2 * Bu + col);
-            }
+            if (next) { n0 = __ldg(next); n1 = __ldg(next + Bu); n2 = __ldg(next + 2 * Bu); }
             LaneX X;
-            {
-                const uint4* src = reinterpret_cast<const uint4*>(xq_rec);
-                const uint4 t0 = __ldg(src), t1 = __ldg(src + 1), t2 = __ldg(src + 2), t3 = __ldg(src + 3),
-                            t4 = __ldg(src + 4);
-                X.hi[0] = t0.x; X.hi[1] = t0.y; X.hi[2] = t0.z; X.hi[3] = t0.w; X.hi[4] = t1.x; X.hi[5] = t1.y;
-                X.mid[0] = t1.z; X.mid[1] = t1.w; X.mid[2] = t2.x; X.mid[3] = t2.y; X.mid[4] = t2.z; X.mid[5] = t2.w;
-                X.lo[0] = t3.x; X.lo[1] = t3.y; X.lo[2] = t3.z; X.lo[3] = t3.w; X.lo[4] = t4.x; X.lo[5] = t4.y;
-                X.step = active ? __uint_as_float(t4.z) : 0.f;
-                X.sum = int(t4.w);
-            }
+            load_lane_x(xq_p + (joint ? lane_col : uint32_t(cg * 32 + lane)) * uint32_t(kXqBytesPerCol),
+                        !joint || lane_in, X);
             float v[8];
             record_values(sm_tab, a, b, h, X, v);
+            if (!joint) {
 #pragma unroll
-            for (int r = 0; r < 8; ++r) acc[r] += v[r];
+                for (int r = 0; r < 8; ++r) acc[r] += v[r];
+                if (++cg == CGf) {  // row group done: fold its eight accumulators into this lane's row
+                    const float t = transpose_partial(red, lane, acc);
+                    if (gi == 0) s0 = t; else if (gi == 1) s1 = t; else s2 = t;
+#pragma unroll
+                    for (int r = 0; r < 8; ++r) acc[r] = 0.f;
+                    cg = 0;
+                    ++gi;
+                }
+            } else {
+                // lane -> (row group, column); lane l then sums, for row l / 4, the columns
+                // k = l % 4, l % 4 + 4, ... of every row group's segment of the buffer
+                __syncwarp();
+#pragma unroll
+                for (int r = 0; r < 8; ++r) red[r * kRedStride + lane] = v[r];
+                __syncwarp();
+                const float* rr = red + (lane >> 2) * kRedStride;
+                for (int k = lane & 3; k < rem; k += 4) {
+                    s0 += rr[k];
+                    if (R > 1) s1 += rr[rem + k];
+                    if (R > 2) s2 += rr[2 * rem + k];
+                }
+            }
         }
-        // row sums, row scale, tail (Sec. 5.1); four lanes per row share the tail
-        float sum = transpose_partial(red, lane, acc);
-        const int row = g * 8 + (lane >> 2);
-        if (row < P.N) {
-            sum *= __ldg(P.row_scales + row);
-            const __half* xh = static_cast<const __half*>(P.x) + 24 * B;
-            const __half* tl = static_cast<const __half*>(P.tail) + size_t(row) * ntail;
-            for (int k = lane & 3; k < ntail; k += 4) sum = fmaf(__half2float(tl[k]), __half2float(xh[k]), sum);
+        // row scale, tail (Sec. 5.1; four lanes per row share the tail), store
+        {
+            const Problem P = problems[p];
+            const int ntail = P.tail ? P.K % 24 : 0;
+            const __half* xh = static_cast<const __half*>(P.x) + 24 * Bu;
+            for (int gk = 0; gk < ng; ++gk) {
+                const int row = (g0 + gk) * 8 + (lane >> 2);
+                float sum = gk == 0 ? s0 : (gk == 1 ? s1 : s2);
+                if (row < P.N) {
+                    sum *= __ldg(P.row_scales + row);
+                    const __half* tl = static_cast<const __half*>(P.tail) + size_t(row) * ntail;
+                    for (int k = lane & 3; k < ntail; k += 4)
+                        sum = fmaf(__half2float(tl[k]), __half2float(xh[k]), sum);
+                }
+                sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
+                sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
+                if (row < P.N && (lane & 3) == 0) P.y[row] = sum;
+            }
         }
-        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
-        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
-        if (row < P.N && (lane & 3) == 0) P.y[row] = sum;
     }
 }
 
@@ -565,7 +628,7 @@ cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, 
     for (int i = 0; i < count; ++i) {
         up[i] = int32_t(units);
         cp[i] = int32_t(cols);
-        units += (problems_host[i].N + 7) / 8;
+        units += problem_units(problems_host[i]);
         cols += problem_blocks(problems_host[i]);
     }
     up[count] = int32_t(units);
@@ -576,16 +639,19 @@ cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, 
     if (e == cudaSuccess && nwarps) {
         // Cut the unit sequence into nwarps contiguous ranges of equal work; a unit costs its number of
         // column groups plus a little for its prologue and epilogue.
-        auto unit_work = [&](int i) { return (long long)((problem_blocks(problems_host[i]) + 31) / 32) * 8 + 2; };
+        auto unit_work = [&](int i) {
+            const int Bi = problem_blocks(problems_host[i]);
+            return (long long)(groups_per_unit(Bi) * (Bi / 32) + (Bi % 32 ? 1 : 0)) * 8 + 2;
+        };
         long long total = 0;
-        for (int i = 0; i < count; ++i) total += unit_work(i) * ((problems_host[i].N + 7) / 8);
+        for (int i = 0; i < count; ++i) total += unit_work(i) * problem_units(problems_host[i]);
         int32_t* wsx = reinterpret_cast<int32_t*>(buf + H->off_warp_start);
         int pi = 0;
         long long before = 0;  // work of matrices 0..pi-1
         for (int w = 0; w < nwarps; ++w) {
             const long long target = total * w / nwarps;
-            while (pi < count - 1 && before + unit_work(pi) * ((problems_host[pi].N + 7) / 8) <= target) {
-                before += unit_work(pi) * ((problems_host[pi].N + 7) / 8);
+            while (pi < count - 1 && before + unit_work(pi) * problem_units(problems_host[pi]) <= target) {
+                before += unit_work(pi) * problem_units(problems_host[pi]);
                 ++pi;
             }
             long long uu = up[pi] + (target - before) / unit_work(pi);
@@ -610,7 +676,7 @@ void single_plan_fill(const Problem& problem, unsigned char* meta_host) {
     memset(meta_host, 0, plan_meta_bytes(1, 0));
     PlanHeader* H = reinterpret_cast<PlanHeader*>(meta_host);
     H->count = 1;
-    H->total_units = (problem.N + 7) / 8;
+    H->total_units = problem_units(problem);
     H->total_cols = problem_blocks(problem);
     H->off_problems = uint32_t(sizeof(PlanHeader));
     H->nwarps = 0;  // no unit ranges: the kernel deals units round-robin
