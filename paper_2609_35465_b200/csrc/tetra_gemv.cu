@@ -493,8 +493,12 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
     const unsigned char* xq_p = xq_all;
     int G = 1;
     uint32_t Bu = 1;
-    bool have_record = false;            // n0..n2 already hold the first record of the unit about to start
-    uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0, n2 = n0;
+    bool have_record = false;            // the ring already holds the first record of the unit about to start
+    // Code records reach the decoder through a per-warp ring in shared memory: two slots of 3 x 512
+    // bytes (one 16-byte part per lane), filled with cp.async one pass ahead, so the prefetch holds
+    // no registers while eight blocks are being decoded.  Each lane reads back only what it copied.
+    const uint32_t ring = sm_tab + uint32_t(kFastBytes) + uint32_t(kUnitWarps * kRedFloats * 4) + uint32_t(warp) * 3072u + uint32_t(lane) * 16u;
+    int pass_parity = 0;
 
     for (; u < u_end; u += u_step) {
         if (u >= p_end) {  // first unit, or the walk has left the matrix: units only go up
@@ -523,7 +527,11 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
 
         if (!have_record) {
             const uint4* first = CGf > 0 ? codes0 + lane : rem_rec;
-            n0 = __ldg(first); n1 = __ldg(first + Bu); n2 = __ldg(first + 2 * Bu);
+            const uint32_t dst = ring + uint32_t(pass_parity * 1536);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst), "l"(first));
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst + 512), "l"(first + Bu));
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst + 1024), "l"(first + 2 * Bu));
+            asm volatile("cp.async.commit_group;");
         }
         have_record = false;
         float s0 = 0.f, s1 = 0.f, s2 = 0.f;  // per row group: this lane's partial row sum (row lane / 4)
@@ -537,7 +545,14 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
         int gi = 0, cg = 0;
         for (int pass = 0; pass < passes; ++pass) {
             const bool joint = pass >= full_passes;
-            const uint4 a = n0, b = n1, h = n2;
+            uint4 a, b, h;
+            {
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                const uint32_t src = ring + uint32_t(pass_parity * 1536);
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "r"(src));
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "r"(src + 512));
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(h.x), "=r"(h.y), "=r"(h.z), "=r"(h.w) : "r"(src + 1024));
+            }
             // prefetch the next pass's record (or the first one of this warp's next unit)
             const uint4* next = nullptr;
             if (pass + 1 < full_passes) {
@@ -549,12 +564,19 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
                 next = codes0 + size_t(u_step) * R * 3 * Bu + lane;
                 have_record = true;
             }
-            if (next) { n0 = __ldg(next); n1 = __ldg(next + Bu); n2 = __ldg(next + 2 * Bu); }
+            if (next) {
+                const uint32_t dst = ring + uint32_t((pass_parity ^ 1) * 1536);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst), "l"(next));
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst + 512), "l"(next + Bu));
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst + 1024), "l"(next + 2 * Bu));
+            }
+            asm volatile("cp.async.commit_group;");
             LaneX X;
             load_lane_x(xq_p + (joint ? lane_col : uint32_t(cg * 32 + lane)) * uint32_t(kXqBytesPerCol),
                         !joint || lane_in, X);
             float v[8];
             record_values(sm_tab, a, b, h, X, v);
+            pass_parity ^= 1;
             if (!joint) {
 #pragma unroll
                 for (int r = 0; r < 8; ++r) acc[r] += v[r];
@@ -697,7 +719,7 @@ cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s) {
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
-    const uint32_t smem = kTableSmemBytes + kUnitWarps * kRedFloats * 4;
+    const uint32_t smem = kTableSmemBytes + kUnitWarps * kRedFloats * 4 + kUnitWarps * 3072;
     if (!attr_set[dev]) {
         e = cudaFuncSetAttribute(k_gemv_units, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
         if (e != cudaSuccess) return e;
