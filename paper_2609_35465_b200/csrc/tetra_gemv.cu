@@ -26,6 +26,8 @@
 
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
+#include <unordered_map>
 
 #include "tetra_device.cuh"
 #include "tetra_launch.h"
@@ -383,14 +385,30 @@ struct PlanHeader {
     int32_t total_cols;   // sum over matrices of words per row
     int32_t nwarps;       // warps the unit ranges were cut for (0: no ranges, units are dealt round-robin)
     uint32_t off_problems, off_unit_prefix, off_col_prefix, off_xq;
-    uint32_t off_warp_start, pad_[3];
+    uint32_t off_warp_start;
+    // fine mode (small lists): a unit is one row group x a slice of the column groups
+    uint32_t off_fine;      // FineInfo[count], 0 in coarse mode
+    uint32_t off_counters;  // int32 per row group: slices of the group that have finished
+    uint32_t off_partials;  // float [row group][slice][8]
+    int32_t total_groups;
+    int32_t pad_[3];
 };
 
-constexpr int kMaxPlanWarps = 8192;  // room reserved for warp_start in a planned list's workspace
+struct FineInfo {
+    int32_t slices;          // column slices per row group
+    int32_t cgs_per_slice;   // column groups per slice (the last slice may hold fewer)
+    int32_t group_prefix;    // row groups of the matrices before this one
+    int32_t partial_prefix;  // floats of partial sums before this matrix
+};
+
+constexpr int kMaxPlanWarps = 8192;    // room reserved for warp_start in a planned list's workspace
+constexpr long long kFineMaxTasks = 65536;  // upper bound of the (row group, column group) pairs of a fine-mode list
+
+static inline long long problem_tasks(const Problem& q);
 
 static size_t plan_meta_bytes(int count, int nwarps) {
     size_t b = sizeof(PlanHeader) + size_t(count) * sizeof(Problem) + 2 * size_t(count + 1) * 4 +
-               (nwarps ? size_t(nwarps + 1) * 4 : 0);
+               (nwarps ? size_t(nwarps + 1) * 4 : 0) + size_t(count) * sizeof(FineInfo);
     return (b + 255) & ~size_t(255);
 }
 
@@ -407,6 +425,23 @@ __host__ __device__ inline int groups_per_unit(int B) {
     const int r = 32 / rem;
     return r < 3 ? r : 3;
 }
+static inline long long problem_tasks(const Problem& q) {
+    return (long long)((q.N + 7) / 8) * ((problem_blocks(q) + 31) / 32);
+}
+// Space for the fine mode is reserved for every list of at most kFineMaxTasks (row group, column group)
+// pairs; the plan then takes the fine mode when the list has at most five such pairs per warp of the
+// grid (measured on B200: below that the coarse units leave most warps idle, above it the fine mode's
+// partial sums and counters cost more than they gain).
+static bool list_may_be_fine(const Problem* problems, int count) {
+    long long tasks = 0;
+    for (int i = 0; i < count; ++i) tasks += problem_tasks(problems[i]);
+    return tasks <= kFineMaxTasks;
+}
+static bool list_is_fine(const Problem* problems, int count, int nwarps) {
+    long long tasks = 0;
+    for (int i = 0; i < count; ++i) tasks += problem_tasks(problems[i]);
+    return tasks <= kFineMaxTasks && tasks <= 5LL * (nwarps ? nwarps : 2048);
+}
 static inline int problem_units(const Problem& q) {
     const int R = groups_per_unit(problem_blocks(q));
     return ((q.N + 7) / 8 + R - 1) / R;
@@ -415,7 +450,13 @@ static inline int problem_units(const Problem& q) {
 size_t grouped_workspace_bytes(const Problem* problems, int count) {
     size_t cols = 0;
     for (int i = 0; i < count; ++i) cols += size_t(problem_blocks(problems[i]));
-    return plan_meta_bytes(count, kMaxPlanWarps) + cols * kXqBytesPerCol;
+    size_t bytes = plan_meta_bytes(count, kMaxPlanWarps) + cols * kXqBytesPerCol;
+    if (list_may_be_fine(problems, count)) {  // counters and partial sums of the fine mode
+        long long groups = 0, tasks = 0;
+        for (int i = 0; i < count; ++i) { groups += (problems[i].N + 7) / 8; tasks += problem_tasks(problems[i]); }
+        bytes = ((bytes + 255) & ~size_t(255)) + size_t(groups) * 4 + 256 + size_t(tasks) * 8 * 4;
+    }
+    return bytes;
 }
 
 // Largest p with prefix[p] <= v (prefix[0] = 0, prefix[count] > v).
@@ -440,6 +481,11 @@ __global__ void __launch_bounds__(256) k_prepare_x(unsigned char* __restrict__ w
         quantise_column(static_cast<const __half*>(P.x), P.K, gc - col_prefix[p], q);
 #pragma unroll
         for (int k = 0; k < 5; ++k) xq[size_t(gc) * 5 + k] = make_uint4(q[4 * k], q[4 * k + 1], q[4 * k + 2], q[4 * k + 3]);
+    }
+    if (H->off_fine) {  // fine mode: the per-row-group arrival counters start every run at zero
+        int32_t* counters = reinterpret_cast<int32_t*>(ws + H->off_counters);
+        for (int g = blockIdx.x * blockDim.x + threadIdx.x; g < H->total_groups; g += gridDim.x * blockDim.x)
+            counters[g] = 0;
     }
 }
 
@@ -625,6 +671,127 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
     }
 }
 
+// Fine mode of the planned list, for lists too small to fill the GPU with coarse units (single
+// matrices, the matrices of one layer): a unit is one row group x a slice of the column groups.
+// Each unit leaves eight partial row sums in the scratch area and bumps its row group's counter; the
+// unit that finds all the other slices done adds them up in slice order (fixed order, no waiting,
+// no floating-point atomics), applies the row scale and the tail, and stores.
+__global__ void __launch_bounds__(kUnitThreads, 1)
+k_gemv_units_fine(const DeviceTables* __restrict__ tab, unsigned char* __restrict__ ws) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    unsigned char* smem = stage_fast_tables(tab, smem_raw);
+    const uint32_t sm_tab = smem_u32(smem);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float* red = reinterpret_cast<float*>(smem + kFastBytes) + warp * kRedFloats;
+    __syncthreads();
+
+    const PlanHeader* H = reinterpret_cast<const PlanHeader*>(ws);
+    const Problem* problems = reinterpret_cast<const Problem*>(ws + H->off_problems);
+    const int32_t* unit_prefix = reinterpret_cast<const int32_t*>(ws + H->off_unit_prefix);
+    const int32_t* col_prefix = reinterpret_cast<const int32_t*>(ws + H->off_col_prefix);
+    const FineInfo* fine = reinterpret_cast<const FineInfo*>(ws + H->off_fine);
+    int32_t* counters = reinterpret_cast<int32_t*>(ws + H->off_counters);
+    float* partials = reinterpret_cast<float*>(ws + H->off_partials);
+    const unsigned char* xq_all = ws + H->off_xq;
+    const int total_units = H->total_units;
+    const uint32_t ring = sm_tab + uint32_t(kFastBytes) + uint32_t(kUnitWarps * kRedFloats * 4) +
+                          uint32_t(warp) * 3072u + uint32_t(lane) * 16u;
+
+    // equal shares of consecutive units per warp (units of a list in fine mode are of similar size)
+    const int gw = blockIdx.x * kUnitWarps + warp, nw = gridDim.x * kUnitWarps;
+    int u = int((long long)total_units * gw / nw);
+    const int u_end = int((long long)total_units * (gw + 1) / nw);
+    int p = -1, p_begin = 0, p_end = 0;
+    Problem P{};
+    FineInfo F{};
+    int CG = 1;
+    uint32_t Bu = 1;
+    const unsigned char* xq_p = xq_all;
+
+    for (; u < u_end; ++u) {
+        if (u >= p_end) {
+            do { ++p; p_end = __ldg(unit_prefix + p + 1); } while (u >= p_end);
+            p_begin = __ldg(unit_prefix + p);
+            P = problems[p];
+            F = fine[p];
+            Bu = uint32_t(P.tail ? P.K / 24 : (P.K + 23) / 24);
+            CG = int((Bu + 31) >> 5);
+            xq_p = xq_all + size_t(__ldg(col_prefix + p)) * kXqBytesPerCol;
+        }
+        const int local = u - p_begin;
+        const int g = local / F.slices, slice = local - g * F.slices;
+        const int c0 = slice * F.cgs_per_slice, c1 = min(CG, c0 + F.cgs_per_slice);
+        const uint4* codes = static_cast<const uint4*>(P.codes) + size_t(g) * 3 * Bu;
+
+        float acc[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) acc[r] = 0.f;
+        {   // first record of the unit into ring slot 0
+            const uint4* first = codes + min(uint32_t(c0 * 32 + lane), Bu - 1);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(ring), "l"(first));
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(ring + 512), "l"(first + Bu));
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(ring + 1024), "l"(first + 2 * Bu));
+            asm volatile("cp.async.commit_group;");
+        }
+        int parity = 0;
+        for (int cg = c0; cg < c1; ++cg) {
+            uint4 a, b, h;
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            {
+                const uint32_t src = ring + uint32_t(parity * 1536);
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "r"(src));
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "r"(src + 512));
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(h.x), "=r"(h.y), "=r"(h.z), "=r"(h.w) : "r"(src + 1024));
+            }
+            if (cg + 1 < c1) {
+                const uint4* next = codes + min(uint32_t((cg + 1) * 32 + lane), Bu - 1);
+                const uint32_t dst = ring + uint32_t((parity ^ 1) * 1536);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst), "l"(next));
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst + 512), "l"(next + Bu));
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst + 1024), "l"(next + 2 * Bu));
+            }
+            asm volatile("cp.async.commit_group;");
+            const uint32_t col = uint32_t(cg * 32 + lane);
+            LaneX X;
+            load_lane_x(xq_p + min(col, Bu - 1) * uint32_t(kXqBytesPerCol), col < Bu, X);
+            float v[8];
+            record_values(sm_tab, a, b, h, X, v);
+#pragma unroll
+            for (int r = 0; r < 8; ++r) acc[r] += v[r];
+            parity ^= 1;
+        }
+        float sum = transpose_partial(red, lane, acc);
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
+        float* mine = partials + F.partial_prefix + (size_t(g) * F.slices + slice) * 8;
+        if ((lane & 3) == 0) mine[lane >> 2] = sum;
+        __threadfence();   // the partial sums are visible before the counter moves
+        __syncwarp();
+        int arrived = 0;
+        if (lane == 0) arrived = atomicAdd(counters + F.group_prefix + g, 1);
+        arrived = __shfl_sync(0xFFFFFFFFu, arrived, 0);
+        if (arrived == F.slices - 1) {  // every slice of this row group is in: finish the rows
+            __threadfence();
+            const int row = g * 8 + lane;
+            if (lane < 8 && row < P.N) {
+                const float* all = partials + F.partial_prefix + size_t(g) * F.slices * 8 + lane;
+                float total = 0.f;
+                for (int k = 0; k < F.slices; ++k) total += __ldcg(all + 8 * k);
+                float res = __ldg(P.row_scales + row) * total;
+                const int ntail = P.tail ? P.K % 24 : 0;
+                const __half* xh = static_cast<const __half*>(P.x) + 24 * Bu;
+                const __half* tl = static_cast<const __half*>(P.tail) + size_t(row) * ntail;
+                for (int k = 0; k < ntail; ++k) res = fmaf(__half2float(tl[k]), __half2float(xh[k]), res);
+                P.y[row] = res;
+            }
+        }
+    }
+}
+
+// grouped_run must know a plan's mode without reading device memory: grouped_plan notes it here.
+static std::mutex g_plan_mu;
+static std::unordered_map<const void*, bool> g_plan_is_fine;
+
 cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, size_t ws_bytes, cudaStream_t s) {
     if (ws_bytes < grouped_workspace_bytes(problems_host, count)) return cudaErrorInvalidValue;
     int sms = 0;
@@ -646,7 +813,39 @@ cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, 
     memcpy(buf + H->off_problems, problems_host, size_t(count) * sizeof(Problem));
     int32_t* up = reinterpret_cast<int32_t*>(buf + H->off_unit_prefix);
     int32_t* cp = reinterpret_cast<int32_t*>(buf + H->off_col_prefix);
+    const bool fine_mode = list_is_fine(problems_host, count, nwarps);
     long long units = 0, cols = 0;
+    if (fine_mode) {
+        // column groups per unit: aim at about four units per warp of the grid
+        long long tasks = 0, groups = 0;
+        for (int i = 0; i < count; ++i) { tasks += problem_tasks(problems_host[i]); groups += (problems_host[i].N + 7) / 8; }
+        const long long want = 4LL * (nwarps ? nwarps : 2048);
+        long long per = tasks / want;
+        if (per < 1) per = 1;
+        H->off_fine = H->off_col_prefix + uint32_t(count + 1) * 4u + (nwarps ? uint32_t(nwarps + 1) * 4u : 0u);
+        FineInfo* fi = reinterpret_cast<FineInfo*>(buf + H->off_fine);
+        size_t xq_end = size_t(H->off_xq);
+        for (int i = 0; i < count; ++i) xq_end += size_t(problem_blocks(problems_host[i])) * kXqBytesPerCol;
+        xq_end = (xq_end + 255) & ~size_t(255);
+        H->off_counters = uint32_t(xq_end);
+        H->off_partials = uint32_t((xq_end + size_t(groups) * 4 + 255) & ~size_t(255));
+        H->total_groups = int32_t(groups);
+        long long gp = 0, pp = 0;
+        for (int i = 0; i < count; ++i) {
+            const int CGi = (problem_blocks(problems_host[i]) + 31) / 32, Gi = (problems_host[i].N + 7) / 8;
+            const int cps = int(per < CGi ? per : CGi);
+            const int slices = (CGi + cps - 1) / cps;
+            fi[i] = FineInfo{slices, cps, int32_t(gp), int32_t(pp)};
+            up[i] = int32_t(units);
+            cp[i] = int32_t(cols);
+            units += (long long)Gi * slices;
+            cols += problem_blocks(problems_host[i]);
+            gp += Gi;
+            pp += (long long)Gi * slices * 8;
+        }
+        nwarps = 0;  // the fine kernel cuts equal shares itself
+        H->nwarps = 0;
+    } else
     for (int i = 0; i < count; ++i) {
         up[i] = int32_t(units);
         cp[i] = int32_t(cols);
@@ -685,6 +884,10 @@ cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, 
     // pageable source: the runtime stages it before returning, so the buffer can be freed
     if (e == cudaSuccess) e = cudaMemcpyAsync(ws_dev, buf, meta, cudaMemcpyHostToDevice, s);
     free(buf);
+    if (e == cudaSuccess) {
+        std::lock_guard<std::mutex> lock(g_plan_mu);
+        g_plan_is_fine[ws_dev] = fine_mode;
+    }
     return e;
 }
 
@@ -723,13 +926,25 @@ cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s) {
     if (!attr_set[dev]) {
         e = cudaFuncSetAttribute(k_gemv_units, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
         if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(k_gemv_units_fine, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (e != cudaSuccess) return e;
         attr_set[dev] = true;
+    }
+    bool fine_mode = false;
+    {
+        std::lock_guard<std::mutex> lock(g_plan_mu);
+        auto it = g_plan_is_fine.find(ws_dev);
+        if (it != g_plan_is_fine.end()) fine_mode = it->second;
     }
     k_prepare_x<<<sms * 2, 256, 0, s>>>(static_cast<unsigned char*>(ws_dev));
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    k_gemv_units<<<sms, kUnitThreads, smem, s>>>(static_cast<const DeviceTables*>(table),
-                                                 static_cast<const unsigned char*>(ws_dev));
+    if (fine_mode)
+        k_gemv_units_fine<<<sms, kUnitThreads, smem, s>>>(static_cast<const DeviceTables*>(table),
+                                                          static_cast<unsigned char*>(ws_dev));
+    else
+        k_gemv_units<<<sms, kUnitThreads, smem, s>>>(static_cast<const DeviceTables*>(table),
+                                                     static_cast<const unsigned char*>(ws_dev));
     return cudaGetLastError();
 }
 

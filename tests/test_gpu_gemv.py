@@ -115,6 +115,32 @@ def test_grouped_launch_one_layer(tt, table, orc):
 
 
 
+@pytest.mark.parametrize("shapes_list", [
+    [(512, 2560, True), (264, 12288, True), (72, 17408, True), (9, 24 * 33, True)],   # a few matrices
+    [(1024, 4096, True)],                                                             # a single one
+    [(33, 24 * 31 + 5, False), (7, 48, True), (1, 24, True)],                         # tiny and ragged
+])
+def test_grouped_small_lists(tt, table, orc, shapes_list):
+    """Small lists run in the planned path's fine mode (one row group x a slice of the column
+    groups per unit, slices summed in fixed order by the last one to finish): every row checked,
+    and a second run of the same plan gives the same bits."""
+    mats = [make_matrix(38, 100 * i + N, N, K, tm) for i, (N, K, tm) in enumerate(shapes_list)]
+    devs = [upload(tt, table, m) for m in mats]
+    problems = tt.make_problems(devs)
+    ws = torch.empty(tt.tetra_grouped_workspace_bytes(problems), dtype=torch.uint8, device="cuda")
+    tt.tetra_gemv_grouped(problems, table, ws)
+    torch.cuda.synchronize()
+    first = [d["y"].cpu().numpy().copy() for d in devs]
+    for d in devs:
+        d["y"].fill_(float("nan"))
+    tt.tetra_gemv_grouped_run(ws, table)
+    torch.cuda.synchronize()
+    for m, d, f in zip(mats, devs, first):
+        y = d["y"].cpu().numpy()[0]
+        assert np.array_equal(y, f[0])
+        assert_gemv_close(y, oracle_product(orc, m, GAIN), "small list %dx%d" % (m["N"], m["K"]))
+
+
 def test_special_inputs(tt, table, orc):
     N, K = 64, 240
     m = make_matrix(35, 1, N, K, True)
