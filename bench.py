@@ -295,6 +295,41 @@ def main():
         dp.run_grouped()
         torch.cuda.synchronize()
 
+        # microseconds per matrix of the single-matrix entry point (tetra_gemv_tail), per shape of a layer:
+        # 12 distinct copies of the shape replayed from a CUDA graph, so no launch re-reads L2-resident codes
+        peak_now = measured_peak()[0]
+        per_matrix = {}
+        for m in model.layer_matrices():
+            one = DevicePass([shapes.Matrix("%s%d" % (m.name, i), m.N, m.K) for i in range(12)], seed=args.seed + 7)
+            for _ in range(2):
+                one.run_per_matrix()
+            gg = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gg, stream=torch.cuda.Stream()):
+                one.run_per_matrix(stream=torch.cuda.current_stream())
+            us = timed(torch, gg.replay, 20, 3, stream) * 1e3 / 12
+            b = one.items[0]["bytes"]
+            per_matrix[m.name] = {"N": m.N, "K": m.K, "us": us, "GBps": b / us / 1e3,
+                                  "weights_per_s": m.N * m.K / us * 1e6, "frac_of_measured_peak": b / us / 1e3 / peak_now,
+                                  "roofline_us": b / peak_now / 1e3}
+            del one, gg
+        out["per_matrix_tetra_gemv"] = per_matrix
+
+        # the other two model sizes, planned-list pass (same kernels; a few repetitions)
+        others = {}
+        for name in ("qwen3-4b", "qwen3-14b"):
+            if name == model.name or args.layers:
+                continue
+            mm = shapes.MODELS[name]
+            od = DevicePass(mm.all_matrices(), seed=args.seed + 11)
+            t = timed(torch, od.run_grouped, 30, 3, stream)
+            others[name] = {"matrices": len(od.items), "algorithmic_bytes": od.algorithmic_bytes, "ms_per_pass": t,
+                            "GBps": od.algorithmic_bytes / (t * 1e-3) / 1e9,
+                            "frac_of_measured_peak": od.algorithmic_bytes / (t * 1e-3) / 1e9 / peak_now,
+                            "weights_per_s": sum(x.N * x.K for x in mm.all_matrices()) / (t * 1e-3)}
+            del od
+            torch.cuda.empty_cache()
+        out["other_models"] = others
+
         # CPU baseline: the oracle on a bounded sample of the same pass, all host cores
         import oracle
         orc = oracle.get()
