@@ -55,6 +55,16 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 }
 
 // ---------------------------------------------------------------------------
+// Programmatic dependent launch.  Every GEMV kernel lets the next kernel of the
+// stream start early (pdl_release) and waits for its own predecessor only when
+// it first touches data a predecessor may have produced (pdl_wait): tables and
+// codes are constants of the model, activations are not.  Both are no-ops for a
+// kernel launched without the attribute.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ---------------------------------------------------------------------------
 // File-order decode (Sec. 3.3, 3.4)
 // ---------------------------------------------------------------------------
 

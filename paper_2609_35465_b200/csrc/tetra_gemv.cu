@@ -246,8 +246,10 @@ __host__ __device__ inline FastSmemLayout fast_smem_layout(int max_blocks) {
 __global__ void __launch_bounds__(kFastThreads, 1)
 k_gemv_fast(const DeviceTables* __restrict__ tab, const Problem single, int batch, int max_blocks) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    pdl_release();
     const FastSmemLayout L = fast_smem_layout(max_blocks);
     unsigned char* smem = stage_fast_tables(tab, smem_raw);
+    pdl_wait();  // x may come from the previous kernel of the stream; the tables above do not
     const uint32_t sm_tab = smem_u32(smem);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float* red = reinterpret_cast<float*>(smem + L.red) + warp * kRedFloats;
@@ -341,6 +343,23 @@ k_gemv_fast(const DeviceTables* __restrict__ tab, const Problem single, int batc
     }
 }
 
+// Launch with programmatic stream serialization allowed: the kernel may start while its predecessor
+// in the stream is still running and synchronises with it through pdl_wait().
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(grid));
+    cfg.blockDim = dim3(unsigned(block));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 static cudaError_t device_sms(int* sms) {
     static int cached[64] = {0};
     int dev = 0;
@@ -367,9 +386,8 @@ cudaError_t launch_gemv_fast(const Problem& single, int batch, int max_blocks, c
     if (L.total > 227u * 1024u) return cudaErrorInvalidValue;
     const int groups = (single.N + 7) / 8;
     const int grid = groups < sms ? groups : sms;
-    k_gemv_fast<<<grid, kFastThreads, L.total, s>>>(static_cast<const DeviceTables*>(table), single, batch,
-                                                    max_blocks);
-    return cudaGetLastError();
+    return launch_pdl(k_gemv_fast, grid, kFastThreads, L.total, s, static_cast<const DeviceTables*>(table), single,
+                      batch, max_blocks);
 }
 
 // ===========================================================================
@@ -470,6 +488,8 @@ __device__ __forceinline__ int find_problem(const int32_t* __restrict__ prefix, 
 }
 
 __global__ void __launch_bounds__(256) k_prepare_x(unsigned char* __restrict__ ws) {
+    pdl_release();
+    pdl_wait();  // the activations (and the plan) may come from the previous kernel of the stream
     const PlanHeader* H = reinterpret_cast<const PlanHeader*>(ws);
     const Problem* problems = reinterpret_cast<const Problem*>(ws + H->off_problems);
     const int32_t* col_prefix = reinterpret_cast<const int32_t*>(ws + H->off_col_prefix);
@@ -509,11 +529,13 @@ constexpr int kUnitWarps = kUnitThreads / 32;
 __global__ void __launch_bounds__(kUnitThreads, 1)
 k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restrict__ ws) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    pdl_release();
     unsigned char* smem = stage_fast_tables(tab, smem_raw);
     const uint32_t sm_tab = smem_u32(smem);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float* red = reinterpret_cast<float*>(smem + kFastBytes) + warp * kRedFloats;
     __syncthreads();  // the only CTA-wide barrier: tables are staged
+    pdl_wait();       // the plan's activation records come from k_prepare_x
 
     const PlanHeader* H = reinterpret_cast<const PlanHeader*>(ws);
     const Problem* problems = reinterpret_cast<const Problem*>(ws + H->off_problems);
@@ -679,11 +701,13 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
 __global__ void __launch_bounds__(kUnitThreads, 1)
 k_gemv_units_fine(const DeviceTables* __restrict__ tab, unsigned char* __restrict__ ws) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    pdl_release();
     unsigned char* smem = stage_fast_tables(tab, smem_raw);
     const uint32_t sm_tab = smem_u32(smem);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float* red = reinterpret_cast<float*>(smem + kFastBytes) + warp * kRedFloats;
     __syncthreads();
+    pdl_wait();  // the plan's activation records and zeroed counters come from k_prepare_x
 
     const PlanHeader* H = reinterpret_cast<const PlanHeader*>(ws);
     const Problem* problems = reinterpret_cast<const Problem*>(ws + H->off_problems);
@@ -936,16 +960,13 @@ cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s) {
         auto it = g_plan_is_fine.find(ws_dev);
         if (it != g_plan_is_fine.end()) fine_mode = it->second;
     }
-    k_prepare_x<<<sms * 2, 256, 0, s>>>(static_cast<unsigned char*>(ws_dev));
-    e = cudaGetLastError();
+    e = launch_pdl(k_prepare_x, sms * 2, 256, 0, s, static_cast<unsigned char*>(ws_dev));
     if (e != cudaSuccess) return e;
     if (fine_mode)
-        k_gemv_units_fine<<<sms, kUnitThreads, smem, s>>>(static_cast<const DeviceTables*>(table),
-                                                          static_cast<unsigned char*>(ws_dev));
-    else
-        k_gemv_units<<<sms, kUnitThreads, smem, s>>>(static_cast<const DeviceTables*>(table),
-                                                     static_cast<const unsigned char*>(ws_dev));
-    return cudaGetLastError();
+        return launch_pdl(k_gemv_units_fine, sms, kUnitThreads, smem, s, static_cast<const DeviceTables*>(table),
+                          static_cast<unsigned char*>(ws_dev));
+    return launch_pdl(k_gemv_units, sms, kUnitThreads, smem, s, static_cast<const DeviceTables*>(table),
+                      static_cast<const unsigned char*>(ws_dev));
 }
 
 }  // namespace tetra
