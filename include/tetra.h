@@ -150,6 +150,19 @@ int tetra_gemv_grouped_run(void *workspace_dev, const void *table, void *stream)
 int tetra_gemv_grouped(const tetra_problem *problems_host, int count, const void *table,
                        void *workspace_dev, size_t workspace_bytes, void *stream);
 
+/* Several activation vectors at once (1 <= batch <= 16): every block is decoded
+ * once and multiplied with all vectors; the contraction over a block's 24
+ * coordinates runs on the tensor cores (int8 x int8 -> int32, exact), the
+ * per-block scale and the accumulation across blocks in float32.  Same result
+ * definition as tetra_gemv_tail.  workspace_dev: 16-byte aligned scratch of at
+ * least tetra_batched_workspace_bytes(N, K) bytes (the vectors' fixed-point
+ * image, and partial results of column chunks that are summed in a fixed
+ * order), private to the call until it completes. */
+size_t tetra_batched_workspace_bytes(int N, int K);
+int tetra_gemv_batched(const void *codes, const float *row_scales, const void *table,
+                       const void *x, float *y, int N, int K, int batch, const void *tail,
+                       void *workspace_dev, size_t workspace_bytes, void *stream);
+
 /* The design the paper describes for its own GPU (Sec. 5.1: a warp per output
  * row, a lane per block, six table loads per block), kept as a comparison arm
  * and a cross-check.  codes: file-order words, row_stride bytes per row

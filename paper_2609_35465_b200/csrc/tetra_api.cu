@@ -187,6 +187,24 @@ int tetra_gemv_grouped(const tetra_problem* problems_host, int count, const void
     return tetra_gemv_grouped_run(workspace_dev, table, stream);
 }
 
+size_t tetra_batched_workspace_bytes(int N, int K) {
+    return (N > 0 && K > 0) ? batched_workspace_bytes(N, (K + 23) / 24) : 0;
+}
+
+int tetra_gemv_batched(const void* codes, const float* row_scales, const void* table, const void* x, float* y, int N,
+                       int K, int batch, const void* tail, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    const int rc = check_gemv(codes, row_scales, table, x, y, N, K, batch);
+    if (rc) return rc;
+    if (!workspace_dev) return TETRA_ERR_NULL;
+    if (!aligned(workspace_dev, 16) || (tail && !aligned(tail, 2))) return TETRA_ERR_ALIGN;
+    const bool tail_mode = tail != nullptr || K % 24 == 0;
+    const int B = tail_mode ? K / 24 : (K + 23) / 24;
+    if (B <= 0 || B > kMaxBlocksPerRow) return TETRA_ERR_SHAPE;
+    if (workspace_bytes < batched_workspace_bytes(N, B)) return TETRA_ERR_SIZE;
+    return cuda_status(launch_gemv_batched(codes, row_scales, table, x, y, N, K, batch, (K % 24) ? tail : nullptr,
+                                           workspace_dev, as_stream(stream)));
+}
+
 int tetra_gemv_paper_design(const void* codes, size_t row_stride, const float* row_scales, const void* table,
                             const void* x, float* y, int N, int K, int batch, const void* tail, void* stream) {
     if (!codes || !row_scales || !table || !x || !y) return TETRA_ERR_NULL;

@@ -109,58 +109,6 @@ constexpr int kRowAccFloats = 2048;            // k_gemv_fast: per-CTA buffer of
 constexpr int kXqBytesPerCol = 80;             // 3 planes x 24 bytes, step, sum
 constexpr uint32_t kXqHi = 0, kXqMid = 24, kXqLo = 48;
 
-// Fixed-point image of one block column of activations (20 words).
-// step = 2^(E-22) with 2^E <= max|x| < 2^(E+1); q_j = rint(x_j / step), |q_j| < 2^23,
-// stored as three byte planes (bits 23..16 signed, 15..8 and 7..0 unsigned), four
-// coordinates per 32-bit word: words 0..5 high, 6..11 middle, 12..17 low plane;
-// word 18 = step (float), word 19 = sum(q_j).  A float16 x_j is held exactly when
-// |x_j| >= 2^(E-12); smaller ones are rounded to a multiple of the step.
-__device__ __forceinline__ void quantise_column(const __half* __restrict__ x, int K, int c, uint32_t out[20]) {
-    float v[24];
-    const int k0 = 24 * c;
-    if (k0 + 24 <= K && ((reinterpret_cast<uintptr_t>(x) & 15) == 0)) {  // 48-byte column, 16-byte aligned
-        const uint4* src = reinterpret_cast<const uint4*>(x + k0);
-#pragma unroll
-        for (int i = 0; i < 3; ++i) {
-            const uint4 u = __ldg(src + i);
-            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const __half2 h = *reinterpret_cast<const __half2*>(&w[j]);
-                v[8 * i + 2 * j] = __low2float(h);
-                v[8 * i + 2 * j + 1] = __high2float(h);
-            }
-        }
-    } else {
-#pragma unroll
-        for (int j = 0; j < 24; ++j) v[j] = k0 + j < K ? __half2float(x[k0 + j]) : 0.f;
-    }
-    float mx = 0.f;
-#pragma unroll
-    for (int j = 0; j < 24; ++j) mx = fmaxf(mx, fabsf(v[j]));
-    const uint32_t e = __float_as_uint(mx) >> 23;  // biased exponent of the largest (finite float16 input)
-    const float step = mx > 0.f ? __uint_as_float((e - 22u) << 23) : 0.f;
-    const float inv = mx > 0.f ? __uint_as_float((276u - e) << 23) : 0.f;
-    int sum = 0;
-#pragma unroll
-    for (int k = 0; k < 6; ++k) {
-        uint32_t hi = 0, mid = 0, lo = 0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int q = __float2int_rn(v[4 * k + i] * inv);
-            sum += q;
-            hi |= (uint32_t(q >> 16) & 0xFFu) << (8 * i);
-            mid |= (uint32_t(q >> 8) & 0xFFu) << (8 * i);
-            lo |= (uint32_t(q) & 0xFFu) << (8 * i);
-        }
-        out[k] = hi;
-        out[6 + k] = mid;
-        out[12 + k] = lo;
-    }
-    out[18] = __float_as_uint(step);
-    out[19] = uint32_t(sum);
-}
-
 struct LaneX {
     uint32_t hi[6];   // bits 23..16 of q (signed), int8 x 4
     uint32_t mid[6];  // bits 15..8 (unsigned)

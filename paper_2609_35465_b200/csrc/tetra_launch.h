@@ -39,6 +39,12 @@ cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, 
 cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s);
 
 
+// 2..16 activation vectors at once (decode once, tensor-core contraction per block); ws holds the
+// vectors' fixed-point image, arrival counters and partial results: batched_workspace_bytes(N, words per row).
+size_t batched_workspace_bytes(int N, int blocks_per_row);
+cudaError_t launch_gemv_batched(const void* codes, const float* row_scales, const void* table, const void* x,
+                                float* y, int N, int K, int batch, const void* tail, void* ws, cudaStream_t s);
+
 // Plan of a single product, for callers that bring their own scratch memory:
 // single_plan_fill writes single_plan_meta_bytes() bytes of plan data to a host
 // buffer; copied to the start of a scratch area of single_plan_scratch_bytes(blocks)

@@ -62,6 +62,9 @@ def lib():
         L.tetra_gemv_paper_design.argtypes = [vp, sz, vp, vp, vp, vp, i32, i32, i32, vp, vp]
         L.tetra_gemv_hostio.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp]
         L.tetra_gemv_grouped_hostio.argtypes = [vp, vp, vp, vp, sz, vp, vp, sz, vp]
+        L.tetra_batched_workspace_bytes.argtypes = [i32, i32]
+        L.tetra_batched_workspace_bytes.restype = sz
+        L.tetra_gemv_batched.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, sz, vp]
         L.tetra_gemv_noalloc.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, vp]
         _lib = L
     return _lib
@@ -217,4 +220,19 @@ def tetra_gemv_noalloc(codes, row_scales, table, x, y, N: int, K: int, tail=None
     Calls on one device share that array, so they must not overlap on the GPU."""
     _check(lib().tetra_gemv_noalloc(_ptr(codes), _ptr(row_scales), _ptr(table), _ptr(x), _ptr(y), N, K,
                                     _ptr(tail), _stream(stream)), "tetra_gemv_noalloc")
+    return y
+
+
+def tetra_batched_workspace_bytes(N: int, K: int) -> int:
+    return lib().tetra_batched_workspace_bytes(N, K)
+
+
+def tetra_gemv_batched(codes, row_scales, table, x, y, N: int, K: int, batch: int, tail=None, workspace=None,
+                       stream=None):
+    """1..16 activation vectors at once: decode once per block, tensor-core contraction per block."""
+    if workspace is None:
+        workspace = torch.empty(tetra_batched_workspace_bytes(N, K), dtype=torch.uint8, device=y.device)
+    _check(lib().tetra_gemv_batched(_ptr(codes), _ptr(row_scales), _ptr(table), _ptr(x), _ptr(y), N, K, batch,
+                                    _ptr(tail), _ptr(workspace), workspace.numel(), _stream(stream)),
+           "tetra_gemv_batched")
     return y
