@@ -155,9 +155,10 @@ int tetra_gemv_grouped(const tetra_problem *problems_host, int count, const void
  * coordinates runs on the tensor cores (int8 x int8 -> int32, exact), the
  * per-block scale and the accumulation across blocks in float32.  Same result
  * definition as tetra_gemv_tail.  workspace_dev: 16-byte aligned scratch of at
- * least tetra_batched_workspace_bytes(N, K) bytes (the vectors' fixed-point
- * image, and partial results of column chunks that are summed in a fixed
- * order), private to the call until it completes. */
+ * least tetra_batched_workspace_bytes(N, K) bytes (partial results of column
+ * ranges, which a second small kernel sums in a fixed order; its contents need
+ * no initialisation), private to the call until it completes.  Two kernel
+ * launches; the result is bit-identical from run to run. */
 size_t tetra_batched_workspace_bytes(int N, int K);
 int tetra_gemv_batched(const void *codes, const float *row_scales, const void *table,
                        const void *x, float *y, int N, int K, int batch, const void *tail,
