@@ -173,6 +173,9 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--layers", type=int, default=0, help="use only the first L layers (profiling runs)")
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary arms and the CPU baseline")
+    ap.add_argument("--batched-only", type=int, default=0, metavar="VECTORS",
+                    help="profiling runs: two rounds of tetra_gemv_batched over 12 copies of the 4096 x 12288 "
+                         "matrix with this many vectors, nothing else, no JSON line")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -200,6 +203,20 @@ def main():
         dist.barrier()
     elif not os.path.exists(tbuild.LIB) and not os.environ.get("TETRA_LIB"):
         tbuild.build()
+
+    if args.batched_only:
+        from paper_2609_35465_b200 import synth, tetra
+        m = shapes.CONFIG4
+        one = DevicePass([shapes.Matrix("sweep%d" % i, m.N, m.K) for i in range(12)], seed=args.seed + 13)
+        ws = torch.empty(tetra.tetra_batched_workspace_bytes(m.N, m.K), dtype=torch.uint8, device="cuda")
+        xb = torch.from_numpy(synth.activations(args.seed + 13, 0, m.K, args.batched_only)).cuda()
+        yb = torch.empty((args.batched_only, m.N), dtype=torch.float32, device="cuda")
+        for _ in range(2):
+            for it in one.items:
+                tetra.tetra_gemv_batched(it["codes"], it["row_scales"], one.table, xb, yb, m.N, m.K,
+                                         args.batched_only, it["tail"], ws)
+        torch.cuda.synchronize()
+        return
 
     model = shapes.MODELS[args.model]
     mats = model.all_matrices()
@@ -313,6 +330,41 @@ def main():
                                   "roofline_us": b / peak_now / 1e3}
             del one, gg
         out["per_matrix_tetra_gemv"] = per_matrix
+
+        # batch sweep on the down_proj shape (N 4096, K 12288): tetra_gemv_batched (decode once, tensor-core
+        # contraction) against one tetra_gemv_tail launch per vector; 12 distinct code copies per CUDA graph
+        from paper_2609_35465_b200 import synth, tetra
+        m = shapes.CONFIG4
+        sweep = {}
+        one = DevicePass([shapes.Matrix("sweep%d" % i, m.N, m.K) for i in range(12)], seed=args.seed + 13)
+        ws = torch.empty(tetra.tetra_batched_workspace_bytes(m.N, m.K), dtype=torch.uint8, device="cuda")
+        for batch in shapes.CONFIG4_BATCHES:
+            xb = torch.from_numpy(synth.activations(args.seed + 13, 0, m.K, batch)).cuda()
+            yb = torch.empty((batch, m.N), dtype=torch.float32, device="cuda")
+
+            def run_batched(stream=None):
+                for it in one.items:
+                    tetra.tetra_gemv_batched(it["codes"], it["row_scales"], one.table, xb, yb, m.N, m.K, batch,
+                                             it["tail"], ws, stream=stream)
+
+            def run_loop(stream=None):
+                for it in one.items:
+                    for v in range(batch):
+                        tetra.tetra_gemv_tail(it["codes"], it["row_scales"], one.table, xb[v], yb[v], m.N, m.K, 1,
+                                              it["tail"], stream=stream)
+            us = {}
+            for name, fn in (("batched", run_batched), ("per_vector", run_loop)):
+                fn()
+                gg = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gg, stream=torch.cuda.Stream()):
+                    fn(stream=torch.cuda.current_stream())
+                us[name] = timed(torch, gg.replay, 10, 3, stream) * 1e3 / 12
+                del gg
+            sweep[str(batch)] = {"batched_us": us["batched"], "per_vector_launches_us": us["per_vector"],
+                                 "us_per_vector": us["batched"] / batch,
+                                 "weights_x_vectors_per_s": m.N * m.K * batch / us["batched"] * 1e6}
+        out["batch_sweep_4096x12288"] = sweep
+        del one, ws
 
         # the other two model sizes, planned-list pass (same kernels; a few repetitions)
         others = {}
