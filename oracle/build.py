@@ -10,23 +10,37 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 SRC = os.path.join(HERE, "tetra_oracle.c")
 HDR = os.path.join(HERE, "tetra_oracle.h")
 LIB = os.path.join(HERE, "libtetra_oracle.so")
+Q4_SRC = os.path.join(HERE, "q4_oracle.c")
+Q4_HDR = os.path.join(HERE, "q4_oracle.h")
+Q4_LIB = os.path.join(HERE, "libq4_oracle.so")
+
+
+def _build_one(lib: str, src: str, hdr: str, force: bool, extra=()) -> str:
+    stale = (
+        force
+        or not os.path.exists(lib)
+        or os.path.getmtime(lib) < max(os.path.getmtime(src), os.path.getmtime(hdr))
+    )
+    if stale:
+        tmp = lib + ".tmp.%d" % os.getpid()
+        cmd = ["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", *extra, "-fopenmp", "-shared", "-fPIC",
+               "-o", tmp, src, "-lm"]
+        subprocess.run(cmd, check=True, cwd=HERE)
+        os.replace(tmp, lib)
+    return lib
 
 
 def build(force: bool = False) -> str:
-    """Build the shared object if it is missing or older than its sources."""
-    stale = (
-        force
-        or not os.path.exists(LIB)
-        or os.path.getmtime(LIB) < max(os.path.getmtime(SRC), os.path.getmtime(HDR))
-    )
-    if stale:
-        tmp = LIB + ".tmp.%d" % os.getpid()
-        cmd = ["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-fopenmp", "-shared", "-fPIC",
-               "-o", tmp, SRC, "-lm"]
-        subprocess.run(cmd, check=True, cwd=HERE)
-        os.replace(tmp, LIB)
-    return LIB
+    """Build the Tetra oracle if it is missing or older than its sources."""
+    return _build_one(LIB, SRC, HDR, force)
+
+
+def build_q4(force: bool = False) -> str:
+    """Build the 4-bit group-quantisation oracle likewise."""
+    # -ffp-contract=off: every product and sum is rounded as written
+    return _build_one(Q4_LIB, Q4_SRC, Q4_HDR, force, extra=("-ffp-contract=off",))
 
 
 if __name__ == "__main__":
     print(build(force=True))
+    print(build_q4(force=True))

@@ -130,3 +130,28 @@ def codes_torch(seed: int, stream: int, N: int, B: int, device="cpu"):
     z = z ^ lsr(z, 31)
     w = lsr(z, 16)
     return w.view(torch.uint8).reshape(n, 8)[:, :6].contiguous().reshape(N, B, 6)
+
+
+# ---------------------------------------------------------------------------
+# 4-bit group-quantised matrices (int4 projections, embedding table, output head)
+# ---------------------------------------------------------------------------
+def q4_nibbles(seed: int, stream: int, N: int, K: int) -> np.ndarray:
+    """uint8 [N, K/2]: two uniform 4-bit weights per byte (weight 2b in the low nibble)."""
+    n = N * (K // 2)
+    w = raw_u64(seed, stream, 11, (n + 7) // 8)
+    return w.view(np.uint8)[:n].reshape(N, K // 2).copy()
+
+
+def q4_scales_offsets(seed: int, stream: int, N: int, groups: int):
+    """float16 [N, groups] each: scale = exp(-5 + 0.3 z) (about a weight range of 0.1 over 15 steps),
+    offset = -scale * (7.5 + 0.5 z'), so that the weights of a group straddle zero."""
+    z = normal(seed, stream, 12, N * groups)
+    z2 = normal(seed, stream, 13, N * groups)
+    scale = np.exp(-5.0 + 0.3 * z).astype(np.float16)
+    offset = (-(scale.astype(np.float64)) * (7.5 + 0.5 * z2)).astype(np.float16)
+    return scale.reshape(N, groups), offset.reshape(N, groups)
+
+
+def token_ids(seed: int, stream: int, count: int, vocab: int) -> np.ndarray:
+    """int32 [count]: uniform row numbers."""
+    return (raw_u64(seed, stream, 14, count) % np.uint64(vocab)).astype(np.int32)
