@@ -60,7 +60,8 @@ def gemv(q, scale, offset, x, N, K, G, batch=1, threads=0, want_termnorm=True):
     """FP64 product; returns (y [batch, N], termnorm [batch, N] or None)."""
     q = np.ascontiguousarray(q, dtype=np.uint8)
     s, o, xx = _u16(scale), _u16(offset), _u16(x)
-    assert q.size == N * (K // 2) and s.size == N * (K // G) == o.size and xx.size == batch * K
+    if not (q.size == N * (K // 2) and s.size == N * (K // G) == o.size and xx.size == batch * K):
+        raise ValueError("q4o_gemv: array sizes do not match N, K, G, batch")
     y = np.zeros((batch, N), dtype=np.float64)
     tn = np.zeros((batch, N), dtype=np.float64) if want_termnorm else None
     rc = _load().q4o_gemv(_p(q), _p(s), _p(o), _p(xx), N, K, G, batch, _p(y), _p(tn) if want_termnorm else None,
