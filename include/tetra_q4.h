@@ -1,0 +1,71 @@
+/*
+ * tetra_q4.h -- C ABI for the 4-bit group-quantised matrices of a served model.
+ *
+ * Besides Tetra blocks, a model file stores some projections as int4 records:
+ * 4-bit weights in groups of 128 along a row, with a float16 scale and a
+ * float16 offset per group (Sec. 4.1, 4.3).  The embedding table and the
+ * output head use the same record with groups of 64 (Sec. 4.4).  The kernel
+ * dequantises each weight with its group's scale and offset and accumulates in
+ * float32 (Sec. 5.1); embedding rows are dequantised on the fly for the input
+ * tokens, and the head is a matrix-vector product over the same table
+ * (Sec. 4.4).
+ *
+ * Conventions are those of tetra.h (status codes, device/host pointers, stream,
+ * validation before launch; a rejected call launches nothing).
+ *
+ * Matrix in file order, as the caller supplies it (the paper leaves these free):
+ *   q       uint8   [N][K/2]   byte b of a row holds weight 2b in its low nibble
+ *                              and weight 2b+1 in its high nibble, values 0..15;
+ *   scale   float16 [N][K/G]   group = k / G;
+ *   offset  float16 [N][K/G];
+ *   weight  w(n,k) = scale[n][k/G] * q(n,k) + offset[n][k/G].
+ * G is 64 or 128 and K a multiple of G (every shape of the three models is).
+ */
+#ifndef TETRA_Q4_H
+#define TETRA_Q4_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TETRA_Q4_MAX_BATCH 8
+#define TETRA_Q4_MAX_K 65536
+
+/* Device layout.  tetra_q4_pack reorders a file-order matrix once (at load) into
+ * the layout the kernels read: rows in strips of 16, each strip a sequence of
+ * 512-byte tiles of 16 rows x 64 weights in which every lane of a warp owns 16
+ * bytes that dequantise, with two logic operations per register, straight
+ * into tensor-core operand registers; then the (scale, offset) pairs as
+ * [strip][group][16 rows].  Rows beyond N are zero.  No bits are added except
+ * that padding: tetra_q4_packed_bytes = ceil(N/16)*16 * (K/2 + 4*K/G).
+ * All three pointers of the source and packed_dev are device memory, 16-byte
+ * aligned; packed_bytes must be at least tetra_q4_packed_bytes(N, K, G)
+ * (0 is returned for a shape that is rejected). */
+size_t tetra_q4_packed_bytes(int N, int K, int G);
+int tetra_q4_pack(const void *q_dev, const void *scale_dev, const void *offset_dev, void *packed_dev,
+                  size_t packed_bytes, int N, int K, int G, void *stream);
+
+/* y[v][n] = sum_k w(n,k) * x[v][k]  for v < batch (Sec. 5.1), 1 <= batch <=
+ * TETRA_Q4_MAX_BATCH.  x_dev: float16 [batch][K], 16-byte aligned; y_dev:
+ * float32 [batch][N].  Products of exact float16 values are accumulated in
+ * float32 (tensor-core m16n8k16, one accumulator per group, then scale and
+ * offset in float32).  One launch, no scratch memory, bit-identical from run
+ * to run. */
+int tetra_q4_gemv(const void *packed_dev, const void *x_dev, float *y_dev, int N, int K, int G, int batch,
+                  void *stream);
+
+/* out[t][k] = float16( fma(scale, q, offset) in float32 ) of row ids[t], for
+ * t < count (Sec. 4.4: rows dequantised for the input tokens).  ids_dev: int32
+ * [count], every id in [0, N) (an id outside it yields a row of zeros and is
+ * not an error the host can see without a copy); out_dev: float16 [count][K],
+ * 8-byte aligned. */
+int tetra_q4_rows(const void *packed_dev, const int32_t *ids_dev, int count, void *out_dev, int N, int K, int G,
+                  void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

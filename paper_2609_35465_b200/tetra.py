@@ -66,6 +66,11 @@ def lib():
         L.tetra_batched_workspace_bytes.restype = sz
         L.tetra_gemv_batched.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, sz, vp]
         L.tetra_gemv_noalloc.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, vp]
+        L.tetra_q4_packed_bytes.argtypes = [i32, i32, i32]
+        L.tetra_q4_packed_bytes.restype = sz
+        L.tetra_q4_pack.argtypes = [vp, vp, vp, vp, sz, i32, i32, i32, vp]
+        L.tetra_q4_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
+        L.tetra_q4_rows.argtypes = [vp, vp, i32, vp, i32, i32, i32, vp]
         _lib = L
     return _lib
 
@@ -236,3 +241,32 @@ def tetra_gemv_batched(codes, row_scales, table, x, y, N: int, K: int, batch: in
                                     _ptr(tail), _ptr(workspace), workspace.numel(), _stream(stream)),
            "tetra_gemv_batched")
     return y
+
+
+# ---------------------------------------------------------------------------
+# 4-bit group-quantised matrices (include/tetra_q4.h)
+# ---------------------------------------------------------------------------
+def tetra_q4_packed_bytes(N: int, K: int, G: int) -> int:
+    n = lib().tetra_q4_packed_bytes(N, K, G)
+    if n == 0:
+        raise TetraError("tetra_q4_packed_bytes: shape rejected (N=%d, K=%d, G=%d)" % (N, K, G))
+    return n
+
+
+def tetra_q4_pack(q, scale, offset, N: int, K: int, G: int, stream=None):
+    """File-order matrix (uint8 [N, K/2], float16 [N, K/G] x 2, all on the device) -> packed device buffer."""
+    packed = torch.empty(tetra_q4_packed_bytes(N, K, G), dtype=torch.uint8, device=q.device)
+    _check(lib().tetra_q4_pack(_ptr(q), _ptr(scale), _ptr(offset), _ptr(packed), packed.numel(), N, K, G,
+                               _stream(stream)), "tetra_q4_pack")
+    return packed
+
+
+def tetra_q4_gemv(packed, x, y, N: int, K: int, G: int, batch: int = 1, stream=None):
+    _check(lib().tetra_q4_gemv(_ptr(packed), _ptr(x), _ptr(y), N, K, G, batch, _stream(stream)), "tetra_q4_gemv")
+    return y
+
+
+def tetra_q4_rows(packed, ids, out, N: int, K: int, G: int, stream=None):
+    _check(lib().tetra_q4_rows(_ptr(packed), _ptr(ids), int(ids.numel()), _ptr(out), N, K, G, _stream(stream)),
+           "tetra_q4_rows")
+    return out

@@ -1,0 +1,124 @@
+"""GPU parity of the 4-bit group-quantised kernels against the FP64 oracle, through the C ABI
+(Sec. 4.1, 4.4, 5.1).  Tolerances as for the Tetra product: relative L2 <= 1e-3 and, per element,
+|delta| <= 1e-3 * sqrt(sum_k (w x)^2) + 1e-6; dequantised rows are bit-exact."""
+import numpy as np
+import pytest
+
+from paper_2609_35465_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+REL_L2, ABS_COEF, ABS_FLOOR = 1e-3, 1e-3, 1e-6
+
+
+def _device_matrix(seed, stream, N, K, G, scale=None, offset=None, q=None):
+    import torch
+    from paper_2609_35465_b200 import tetra
+    q = synth.q4_nibbles(seed, stream, N, K) if q is None else q
+    s, o = synth.q4_scales_offsets(seed, stream, N, K // G)
+    scale = s if scale is None else scale
+    offset = o if offset is None else offset
+    packed = tetra.tetra_q4_pack(torch.from_numpy(q).cuda(), torch.from_numpy(scale).cuda(),
+                                 torch.from_numpy(offset).cuda(), N, K, G)
+    return q, scale, offset, packed
+
+
+def _check_gemv(q, scale, offset, packed, x, N, K, G, batch):
+    import torch
+    from oracle import q4 as oq
+    from paper_2609_35465_b200 import tetra
+    y = torch.full((batch, N), float("nan"), dtype=torch.float32, device="cuda")
+    tetra.tetra_q4_gemv(packed, torch.from_numpy(x).cuda(), y, N, K, G, batch)
+    got = y.cpu().numpy().astype(np.float64)
+    want, tn = oq.gemv(q, scale, offset, x, N, K, G, batch)
+    assert np.isfinite(got).all()
+    rel = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-300)
+    assert rel <= REL_L2, rel
+    bound = ABS_COEF * tn + ABS_FLOOR
+    worst = np.max(np.abs(got - want) / bound)
+    assert worst <= 1.0, worst
+    return rel, worst
+
+
+@pytest.mark.parametrize("N,K,G,batch", [
+    (16, 128, 128, 1), (16, 64, 64, 1), (64, 1024, 128, 1), (37, 1152, 128, 1), (1, 256, 64, 1),
+    (1024, 4096, 128, 1), (2560, 9728, 128, 1), (300, 4096, 64, 1), (512, 17408, 128, 1),
+    (129, 2560, 64, 3), (256, 4096, 128, 8), (2048, 5120, 64, 5),
+])
+def test_q4_gemv_matches_oracle(N, K, G, batch):
+    q, s, o, packed = _device_matrix(21, N + K, N, K, G)
+    x = synth.activations(21, 5, K, batch)
+    _check_gemv(q, s, o, packed, x, N, K, G, batch)
+
+
+def test_q4_gemv_extreme_nibbles_and_scales():
+    """All-15 and all-0 weights, large offsets against small scales, float16-subnormal scales."""
+    N, K, G = 48, 1024, 128
+    x = synth.activations(22, 1, K, 2)
+    for fill in (0x00, 0xFF, 0x0F, 0xF0):
+        q = np.full((N, K // 2), fill, dtype=np.uint8)
+        q_, s, o, packed = _device_matrix(22, 2, N, K, G, q=q)
+        _check_gemv(q, s, o, packed, x, N, K, G, 2)
+    s = np.full((N, K // G), 6e-8, dtype=np.float16)  # subnormal
+    o = np.full((N, K // G), 0.75, dtype=np.float16)
+    q, s, o, packed = _device_matrix(22, 3, N, K, G, scale=s, offset=o)
+    _check_gemv(q, s, o, packed, x, N, K, G, 2)
+
+
+def test_q4_gemv_is_deterministic_and_ignores_other_vectors():
+    import torch
+    from paper_2609_35465_b200 import tetra
+    N, K, G = 700, 4096, 128
+    q, s, o, packed = _device_matrix(23, 1, N, K, G)
+    x = torch.from_numpy(synth.activations(23, 1, K, 4)).cuda()
+    y1 = torch.empty((4, N), dtype=torch.float32, device="cuda")
+    y2 = torch.empty((4, N), dtype=torch.float32, device="cuda")
+    tetra.tetra_q4_gemv(packed, x, y1, N, K, G, 4)
+    tetra.tetra_q4_gemv(packed, x, y2, N, K, G, 4)
+    assert torch.equal(y1, y2)
+    y3 = torch.empty((1, N), dtype=torch.float32, device="cuda")
+    tetra.tetra_q4_gemv(packed, x[2:3].contiguous(), y3, N, K, G, 1)
+    assert torch.equal(y3[0], y1[2])  # a vector's result does not depend on its neighbours in the batch
+
+
+@pytest.mark.parametrize("N,K,G", [(100, 256, 64), (151936, 1024, 64), (50, 2560, 128)])
+def test_q4_rows_bit_exact(N, K, G):
+    import torch
+    from oracle import q4 as oq
+    from paper_2609_35465_b200 import tetra
+    rows = min(N, 4096)  # the oracle side only needs the rows that are looked up
+    ids = synth.token_ids(24, 1, 33, N)
+    ids[0], ids[1] = 0, N - 1
+    q = synth.q4_nibbles(24, N, N, K)
+    s, o = synth.q4_scales_offsets(24, N, N, K // G)
+    s[ids[2], 0] = np.float16(6e-8)  # a subnormal scale on a row that is looked up
+    packed = tetra.tetra_q4_pack(torch.from_numpy(q).cuda(), torch.from_numpy(s).cuda(), torch.from_numpy(o).cuda(),
+                                 N, K, G)
+    out = torch.full((len(ids), K), float("nan"), dtype=torch.float16, device="cuda")
+    tetra.tetra_q4_rows(packed, torch.from_numpy(ids).cuda(), out, N, K, G)
+    del rows
+    want = oq.rows(q, s, o, ids, N, K, G)
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), want.view(np.uint16))
+
+
+def test_q4_argument_checks():
+    import torch
+    from paper_2609_35465_b200 import tetra
+    N, K, G = 32, 256, 64
+    q, s, o, packed = _device_matrix(25, 1, N, K, G)
+    x = torch.zeros((1, K), dtype=torch.float16, device="cuda")
+    y = torch.zeros((1, N), dtype=torch.float32, device="cuda")
+    with pytest.raises(tetra.TetraError):
+        tetra.tetra_q4_gemv(packed, x, y, N, K, 96, 1)  # group size
+    with pytest.raises(tetra.TetraError):
+        tetra.tetra_q4_gemv(packed, x, y, N, 200, 64, 1)  # K not a multiple of G
+    with pytest.raises(tetra.TetraError):
+        tetra.tetra_q4_gemv(packed, x, y, N, K, G, 9)  # batch
+    with pytest.raises(tetra.TetraError):
+        tetra.tetra_q4_packed_bytes(0, K, G)
+    out = torch.zeros((0, K), dtype=torch.float16, device="cuda")
+    tetra.tetra_q4_rows(packed, torch.zeros(0, dtype=torch.int32, device="cuda"), out, N, K, G)  # empty: no launch
+    ids = torch.tensor([5, -1, N], dtype=torch.int32, device="cuda")  # ids outside the table give zero rows
+    out = torch.full((3, K), 1.0, dtype=torch.float16, device="cuda")
+    tetra.tetra_q4_rows(packed, ids, out, N, K, G)
+    assert torch.count_nonzero(out[1:]) == 0 and torch.count_nonzero(out[0]) > 0
