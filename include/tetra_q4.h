@@ -35,12 +35,13 @@ extern "C" {
 #define TETRA_Q4_MAX_K 65536
 
 /* Device layout.  tetra_q4_pack reorders a file-order matrix once (at load) into
- * the layout the kernels read: rows in strips of 16, each strip a sequence of
- * 512-byte tiles of 16 rows x 64 weights in which every lane of a warp owns 16
- * bytes that dequantise, with two logic operations per register, straight
- * into tensor-core operand registers; then the (scale, offset) pairs as
- * [strip][group][16 rows].  Rows beyond N are zero.  No bits are added except
- * that padding: tetra_q4_packed_bytes = ceil(N/16)*16 * (K/2 + 4*K/G).
+ * the layout the kernels read: rows in strips of 32, and for every (strip,
+ * group) one contiguous chunk: 512-byte tiles of 16 rows x 64 weights in which
+ * every lane of a warp owns 16 bytes that dequantise, with five logic
+ * operations per four registers, straight into tensor-core operand registers,
+ * followed by the group's 32 (scale, offset) pairs.  Rows beyond N are zero.  No
+ * bits are added except that padding:
+ * tetra_q4_packed_bytes = ceil(N/32)*32 * (K/2 + 4*K/G).
  * All three pointers of the source and packed_dev are device memory, 16-byte
  * aligned; packed_bytes must be at least tetra_q4_packed_bytes(N, K, G)
  * (0 is returned for a shape that is rejected). */

@@ -26,36 +26,42 @@
 namespace tetra {
 namespace {
 
-constexpr int kQ4Threads = 512;
+#ifndef TETRA_Q4_THREADS
+#define TETRA_Q4_THREADS 512
+#define TETRA_Q4_CTAS 1
+#endif
+constexpr int kQ4Threads = TETRA_Q4_THREADS;
+constexpr int kQ4CtasPerSm = TETRA_Q4_CTAS;
 constexpr int kQ4Warps = kQ4Threads / 32;
 
-// Packed layout (uint4 units): tile (strip, kt) at (strip * KT + kt) * 32 + lane, KT = K / 64; lane = 4 g + t
-// owns four words m = 0..3; word m, nibbles n0..n7 (n_i at bits 4 i), weights of columns
-// c = 64 kt + 16 t + 4 m + {0,1,2,3}:
-//     n0, n4 = row g,     c + 0, c + 1        n1, n5 = row g,     c + 2, c + 3
-//     n2, n6 = row g + 8, c + 0, c + 1        n3, n7 = row g + 8, c + 2, c + 3
-// After the tiles: (scale, offset) half2 records at so_base + (strip * groups + group) * 16 + row.
-__host__ __device__ inline size_t q4_weight_bytes(int strips, int K) { return size_t(strips) * (K / 64) * 512; }
+// Packed layout.  Rows are taken in strips of 32, columns in groups of G; the data of (strip, group) is one
+// contiguous chunk of CH = (G / 64) * 1024 + 128 bytes at (strip * groups + group) * CH:
+//   for each 64-column tile j of the group, two 512-byte sub-tiles h = 0, 1 (rows 16 h .. 16 h + 15 of the
+//   strip) at j * 1024 + h * 512, in which lane = 4 g + t of a warp owns 16 bytes = four words m = 0..3; word m
+//   holds, as nibbles n0..n7 (n_i at bits 4 i), the weights of columns c = 64 j + 16 t + 4 m + {0,1,2,3}:
+//       n0, n4 = row g,     c + 0, c + 1        n1, n5 = row g,     c + 2, c + 3
+//       n2, n6 = row g + 8, c + 0, c + 1        n3, n7 = row g + 8, c + 2, c + 3      (rows within the sub-tile)
+//   then 32 (scale, offset) float16 pairs, one per row of the strip.
+// A warp streams whole chunks; nothing else of the matrix is read.
+__host__ __device__ constexpr int q4_chunk_bytes(int G) { return (G / 64) * 1024 + 128; }
 
 __global__ void __launch_bounds__(256) k_q4_pack(const uint8_t* __restrict__ q, const __half* __restrict__ scale,
                                                  const __half* __restrict__ offset, uint32_t* __restrict__ packed,
                                                  int N, int K, int G) {
-    const int strips = (N + 15) / 16, KT = K / 64, groups = K / G;
-    const size_t words = size_t(strips) * KT * 128;
-    const size_t so_words = size_t(strips) * groups * 16;
-    uint32_t* so = packed + words;
-    for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < words + so_words;
-         i += size_t(gridDim.x) * blockDim.x) {
-        if (i < words) {
-            const int m = int(i & 3), lane = int((i >> 2) & 31);
-            const size_t tile = i >> 7;
-            const int kt = int(tile % KT), strip = int(tile / KT);
+    const int strips = (N + 31) / 32, groups = K / G, chunk_words = q4_chunk_bytes(G) / 4, tile_words = (G / 64) * 256;
+    const size_t total = size_t(strips) * groups * chunk_words;
+    for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < total; i += size_t(gridDim.x) * blockDim.x) {
+        const int wi = int(i % chunk_words);
+        const size_t sg = i / chunk_words;
+        const int group = int(sg % groups), strip = int(sg / groups);
+        uint32_t w = 0;
+        if (wi < tile_words) {
+            const int m = wi & 3, lane = (wi >> 2) & 31, h = (wi >> 7) & 1, j = wi >> 8;
             const int g = lane >> 2, t = lane & 3;
-            const int c = 64 * kt + 16 * t + 4 * m;  // multiple of 4: two whole bytes per row
-            uint32_t w = 0;
+            const int c = group * G + 64 * j + 16 * t + 4 * m;  // multiple of 4: two whole bytes per row
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                const int row = 16 * strip + g + 8 * half;
+                const int row = 32 * strip + 16 * h + g + 8 * half;
                 if (row < N) {
                     const uint8_t* src = q + size_t(row) * (K / 2) + c / 2;
                     const uint32_t b0 = src[0], b1 = src[1];  // b0 = weights c, c+1; b1 = c+2, c+3
@@ -65,20 +71,14 @@ __global__ void __launch_bounds__(256) k_q4_pack(const uint8_t* __restrict__ q, 
                          (n_c3 << (20 + 8 * half));
                 }
             }
-            packed[i] = w;
         } else {
-            const size_t j = i - words;
-            const int r = int(j & 15);
-            const size_t sg = j >> 4;
-            const int group = int(sg % groups), strip = int(sg / groups);
-            const int row = 16 * strip + r;
-            uint32_t v = 0;
+            const int row = 32 * strip + (wi - tile_words);
             if (row < N) {
                 const size_t at = size_t(row) * groups + group;
-                v = uint32_t(__half_as_ushort(scale[at])) | (uint32_t(__half_as_ushort(offset[at])) << 16);
+                w = uint32_t(__half_as_ushort(scale[at])) | (uint32_t(__half_as_ushort(offset[at])) << 16);
             }
-            so[j] = v;
         }
+        packed[i] = w;
     }
 }
 
@@ -93,6 +93,16 @@ __device__ __forceinline__ uint32_t lop_and_or(uint32_t a, uint32_t mask, uint32
     asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(magic));  // (a & mask) | magic
     return r;
 }
+__device__ __forceinline__ void q4_lds128(uint32_t saddr, uint32_t (&v)[4]) {
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(saddr));
+}
+__device__ __forceinline__ void q4_cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+template <int PENDING>
+__device__ __forceinline__ void q4_cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
+}
 
 __device__ __forceinline__ void team_barrier(int team, int team_warps) {
     if (team_warps == 1)
@@ -101,32 +111,86 @@ __device__ __forceinline__ void team_barrier(int team, int team_warps) {
         asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(team_warps * 32) : "memory");
 }
 
-// A team of S warps (S a power of two, 1..16) owns a strip of 16 rows at a time and splits its groups:
-// warp p of the team takes groups p, p + S, ...  Per group: TPG = G / 64 tiles, four MMAs each, into one
-// accumulator; then the bias correction, scale and offset.  At the end of a strip the team's warps add
-// their sums through shared memory (two buffers, one named barrier per strip).
-template <int G>
-__global__ void __launch_bounds__(kQ4Threads, 2)
-k_q4_gemv(const uint4* __restrict__ packed, const __half* __restrict__ x, float* __restrict__ y, int N, int K,
+// A team of S warps (S a power of two, 1..16) owns a strip of 32 rows at a time and splits its groups: warp p
+// of the team takes groups p, p + S, ...  The warp's chunks, across all its strips, form one stream that it
+// copies into a ring of DEPTH slots in shared memory with cp.async, DEPTH - 1 chunks ahead.  Per chunk: the
+// accumulators of the two 16-row sub-tiles start at minus the group's sum(bias_k x_k), every 64-column tile
+// adds four MMAs per sub-tile (the activations' B fragments are shared by both), then
+//     acc += scale * D + offset * sum_group(x).
+// At the end of a strip the team's warps add their sums through shared memory (S > 1) and store.
+// Addresses advance by running pointers: the loop body is dequantise, multiply, scale.
+// First MMA of a group: the accumulator starts from c (minus the group's bias sums).
+__device__ __forceinline__ void mma_f16_first(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1, float c_even,
+                                              float c_odd) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%10,%11};"
+                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(c_even), "f"(c_odd));
+}
+
+// XS: the activations are staged in shared memory (rows padded by 16 bytes so that the eight vectors' reads
+// fall into different banks); otherwise they are read through L1.
+template <int G, int DEPTH, bool XS>
+__global__ void __launch_bounds__(kQ4Threads, kQ4CtasPerSm)
+k_q4_gemv(const unsigned char* __restrict__ packed, const __half* __restrict__ x, float* __restrict__ y, int N, int K,
           int batch, int S) {
-    constexpr int TPG = G / 64;
+    constexpr int TPG = G / 64, CH = q4_chunk_bytes(G), PIECES = CH / 16;
     extern __shared__ __align__(16) unsigned char q4_smem[];
-    const int groups = K / G, KT = K / 64, strips = (N + 15) / 16;
-    float2* gs = reinterpret_cast<float2*>(q4_smem);                                // [groups][8]: (sum x, sum bias x)
-    float* red = reinterpret_cast<float*>(q4_smem + size_t(groups) * 64);           // [2][warps][128]
-    const uint32_t* so = reinterpret_cast<const uint32_t*>(packed + size_t(strips) * KT * 32);
+    const int groups = K / G, strips = (N + 31) / 32;
+    float2* gs = reinterpret_cast<float2*>(q4_smem);                        // [groups][8]: (sum x, -sum bias x)
+    float* red = reinterpret_cast<float*>(q4_smem + size_t(groups) * 64);   // [warps][256]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ring = smem_u32(q4_smem + size_t(groups) * 64 + kQ4Warps * 1024) + uint32_t(warp) * (DEPTH * CH);
+    unsigned char* xs_base = q4_smem + size_t(groups) * 64 + kQ4Warps * 1024 + size_t(kQ4Warps) * DEPTH * CH;
+    const uint32_t xs_stride = uint32_t(K) * 2u + 16u;  // bytes per staged vector
+    const uint32_t ring_end = ring + DEPTH * CH;
     const int g = lane >> 2, t = lane & 3;
     pdl_release();
-    pdl_wait();  // x may come from the preceding kernel
 
-    // per (group, vector): sum of x and of bias_k x_k, bias 1024 for k % 4 in {0, 1}, 64 for {2, 3}
+    const int teams = kQ4Warps / S, team = warp / S, p = warp % S;
+    const int cnt = p < groups ? (groups - p + S - 1) / S : 0;  // chunks of this warp per strip
+    const int strip0 = blockIdx.x * teams + team, strip_step = gridDim.x * teams;
+    const int my_strips = strip0 < strips ? (strips - strip0 + strip_step - 1) / strip_step : 0;
+    // fetch cursor over the warp's stream of chunks (all its strips, one after the other)
+    const unsigned char* f_src = packed + (size_t(strip0) * groups + p) * CH + lane * 16;
+    const uint32_t f_wrap_chunks = uint32_t(strip_step) * uint32_t(groups) - uint32_t(cnt > 0 ? cnt - 1 : 0) * uint32_t(S);
+    int f_left = my_strips * cnt, f_in_strip = cnt;
+    uint32_t f_dst = ring + lane * 16;
+    auto fetch = [&]() {
+        if (f_left > 0) {
+#pragma unroll
+            for (int i = 0; i < (PIECES + 31) / 32; ++i)
+                if ((i + 1) * 32 <= PIECES || lane < PIECES - i * 32) q4_cp_async16(f_dst + i * 512, f_src + i * 512);
+            --f_left;
+            if (--f_in_strip == 0) {
+                f_in_strip = cnt;
+                f_src += size_t(f_wrap_chunks) * CH;
+            } else {
+                f_src += size_t(uint32_t(S)) * CH;
+            }
+        }
+        f_dst += CH;
+        if (f_dst >= ring_end) f_dst -= DEPTH * CH;
+        asm volatile("cp.async.commit_group;" ::: "memory");  // one group per call, empty or not
+    };
+#pragma unroll
+    for (int i = 0; i < DEPTH - 1; ++i) fetch();  // the weights do not depend on the preceding kernel
+
+    pdl_wait();  // x may come from the preceding kernel
+    if (XS) {
+        for (int i = threadIdx.x; i < batch * (K / 8); i += kQ4Threads) {
+            const int v = i / (K / 8), c8 = i % (K / 8);
+            *reinterpret_cast<uint4*>(xs_base + size_t(v) * xs_stride + size_t(c8) * 16) =
+                __ldg(reinterpret_cast<const uint4*>(x + size_t(v) * K) + c8);
+        }
+    }
+    // per (group, vector): sum of x and minus the sum of bias_k x_k, bias 1024 for k % 4 in {0, 1}, 64 for {2, 3}
     for (int task = threadIdx.x; task < groups * 8; task += kQ4Threads) {
         const int v = task & 7, gi = task >> 3;
         float sx = 0.f, sb = 0.f;
         if (v < batch) {
             const uint2* src = reinterpret_cast<const uint2*>(x + size_t(v) * K + size_t(gi) * G);
             float lo = 0.f, hi = 0.f;  // k % 4 in {0, 1} / {2, 3}
+#pragma unroll 4
             for (int i = 0; i < G / 4; ++i) {
                 const uint2 u = __ldg(src + i);
                 const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&u.x));
@@ -135,109 +199,142 @@ k_q4_gemv(const uint4* __restrict__ packed, const __half* __restrict__ x, float*
                 hi += b.x + b.y;
             }
             sx = lo + hi;
-            sb = 1024.f * lo + 64.f * hi;
+            sb = -(1024.f * lo + 64.f * hi);
         }
         gs[task] = make_float2(sx, sb);
     }
     __syncthreads();
 
-    const int teams = kQ4Warps / S, team = warp / S, p = warp % S;
-    const __half* xv = x + size_t(g) * K + 16 * t;  // vector g (columns of B), this lane's 16 activations per tile
-    const bool has_x = g < batch;
-    int buf = 0;
-    for (int strip = blockIdx.x * teams + team; strip < strips; strip += gridDim.x * teams) {
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        const uint4* wrow = packed + size_t(strip) * KT * 32 + lane;
-        const uint32_t* sorow = so + size_t(strip) * groups * 16 + g;
-        // software pipeline over this warp's groups: the next group's weights are in flight during the MMAs
-        uint4 wn[TPG];
-        uint32_t so0n = 0, so1n = 0;
-        if (p < groups) {
+    // column g of B is vector g; columns at or beyond batch are never stored, so they may hold any vector
+    const uint32_t x_vec = uint32_t(g < batch ? g : batch - 1);
+    // this lane's 16 activations of the first tile of group p: an offset in halves (global) or a shared address
+    const uint32_t x_lane = XS ? smem_u32(xs_base) + x_vec * xs_stride + (16u * t + uint32_t(p) * G) * 2u
+                               : x_vec * uint32_t(K) + 16u * t + uint32_t(p) * G;
+    const uint32_t gs_lane = smem_u32(gs) + uint32_t(p) * 64 + uint32_t(t) * 16;
+    uint32_t chunk = ring;
+    int strip = strip0;
+    for (int si = 0; si < my_strips; ++si, strip += strip_step) {
+        float acc[2][4];
 #pragma unroll
-            for (int j = 0; j < TPG; ++j) wn[j] = __ldcs(wrow + size_t(p * TPG + j) * 32);
-            so0n = __ldg(sorow + p * 16);
-            so1n = __ldg(sorow + p * 16 + 8);
-        }
-        for (int gi = p; gi < groups; gi += S) {
-            uint4 w[TPG];
+        for (int h = 0; h < 2; ++h)
 #pragma unroll
-            for (int j = 0; j < TPG; ++j) w[j] = wn[j];
-            const uint32_t so0 = so0n, so1 = so1n;
-            if (gi + S < groups) {
-#pragma unroll
-                for (int j = 0; j < TPG; ++j) wn[j] = __ldcs(wrow + size_t((gi + S) * TPG + j) * 32);
-                so0n = __ldg(sorow + (gi + S) * 16);
-                so1n = __ldg(sorow + (gi + S) * 16 + 8);
-            }
-            float d[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int i = 0; i < 4; ++i) acc[h][i] = 0.f;
+        uint32_t xo = x_lane;
+        uint32_t gsp = gs_lane;
+        for (int idx = 0; idx < cnt; ++idx) {
+            uint32_t cs[4];  // (sum x, -sum bias x) of vectors 2 t, 2 t + 1
+            q4_lds128(gsp, cs);
+            fetch();                        // refill the slot consumed last
+            q4_cp_async_wait<DEPTH - 1>();  // this chunk has landed
+            __syncwarp();
+            float d[2][4];
 #pragma unroll
             for (int j = 0; j < TPG; ++j) {
-                uint4 xa = make_uint4(0, 0, 0, 0), xb = make_uint4(0, 0, 0, 0);
-                if (has_x) {
-                    const uint4* xs = reinterpret_cast<const uint4*>(xv + size_t(gi * TPG + j) * 64);
-                    xa = __ldg(xs);
-                    xb = __ldg(xs + 1);
-                }
-                const uint32_t xr[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-                const uint32_t ww[4] = {w[j].x, w[j].y, w[j].z, w[j].w};
+                uint32_t xr[8];
+                if (XS) {
+                    uint32_t lo[4], hi[4];
+                    q4_lds128(xo + 128 * j, lo);
+                    q4_lds128(xo + 128 * j + 16, hi);
 #pragma unroll
-                for (int m = 0; m < 4; ++m) {
-                    const uint32_t w8 = ww[m] >> 8;
-                    uint32_t a[4];
-                    a[0] = lop_and_or(ww[m], 0x000F000Fu, 0x64006400u);  // row g,     columns c, c+1   (1024 + n)
-                    a[1] = lop_and_or(w8, 0x000F000Fu, 0x64006400u);     // row g + 8, columns c, c+1
-                    a[2] = lop_and_or(ww[m], 0x00F000F0u, 0x54005400u);  // row g,     columns c+2, c+3 (64 + n)
-                    a[3] = lop_and_or(w8, 0x00F000F0u, 0x54005400u);     // row g + 8, columns c+2, c+3
-                    mma_f16(d, a, xr[2 * m], xr[2 * m + 1]);
+                    for (int i = 0; i < 4; ++i) {
+                        xr[i] = lo[i];
+                        xr[4 + i] = hi[i];
+                    }
+                } else {
+                    const uint4* xg = reinterpret_cast<const uint4*>(x + xo) + 8 * j;  // L1-resident activations
+                    const uint4 xa = __ldg(xg);
+                    const uint4 xb = __ldg(xg + 1);
+                    xr[0] = xa.x; xr[1] = xa.y; xr[2] = xa.z; xr[3] = xa.w;
+                    xr[4] = xb.x; xr[5] = xb.y; xr[6] = xb.z; xr[7] = xb.w;
+                }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t ww[4];
+                    q4_lds128(chunk + j * 1024 + h * 512 + lane * 16, ww);
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) {
+                        uint32_t a[4];
+                        const uint32_t w8 = ww[m] >> 8;
+                        a[0] = lop_and_or(ww[m], 0x000F000Fu, 0x64006400u);  // row g,     columns c, c+1   (1024 + n)
+                        a[1] = lop_and_or(w8, 0x000F000Fu, 0x64006400u);     // row g + 8, columns c, c+1
+                        a[2] = lop_and_or(ww[m], 0x00F000F0u, 0x54005400u);  // row g,     columns c+2, c+3 (64 + n)
+                        a[3] = lop_and_or(w8, 0x00F000F0u, 0x54005400u);     // row g + 8, columns c+2, c+3
+                        if (j == 0 && m == 0)
+                            mma_f16_first(d[h], a, xr[0], xr[1], __uint_as_float(cs[1]), __uint_as_float(cs[3]));
+                        else
+                            mma_f16(d[h], a, xr[2 * m], xr[2 * m + 1]);
+                    }
                 }
             }
-            // this lane's results: rows g (i = 0, 1) and g + 8 (i = 2, 3), vectors 2 t + (i & 1)
-            const float4 cs = *reinterpret_cast<const float4*>(gs + gi * 8 + 2 * t);  // (sx, sb) of vectors 2t, 2t+1
-            const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&so0));  // (scale, offset) of row g
-            const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&so1));  // of row g + 8
-            acc[0] += r0.x * (d[0] - cs.y) + r0.y * cs.x;
-            acc[1] += r0.x * (d[1] - cs.w) + r0.y * cs.z;
-            acc[2] += r1.x * (d[2] - cs.y) + r1.y * cs.x;
-            acc[3] += r1.x * (d[3] - cs.w) + r1.y * cs.z;
-        }
-        // team sum in warp order, then store: element e = 4 lane + i is (row g + 8 (i / 2), vector 2 t + (i % 2))
-        float* mine = red + (size_t(buf) * kQ4Warps + warp) * 128;
-        *reinterpret_cast<float4*>(mine + 4 * lane) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-        team_barrier(team, S);
-        const float* first = red + (size_t(buf) * kQ4Warps + team * S) * 128;
-        for (int e = p * 32 + lane; e < 128; e += S * 32) {
-            const int el = e >> 2, i = e & 3;
-            const int row = 16 * strip + (el >> 2) + 8 * (i >> 1), v = 2 * (el & 3) + (i & 1);
-            if (row < N && v < batch) {
-                float total = 0.f;
-                for (int k = 0; k < S; ++k) total += first[k * 128 + e];
-                y[size_t(v) * N + row] = total;
+            // this lane's results: rows 16 h + g (i = 0, 1) and 16 h + g + 8 (i = 2, 3), vectors 2 t + (i & 1)
+            const float sx_even = __uint_as_float(cs[0]), sx_odd = __uint_as_float(cs[2]);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t so0 = lds32(chunk + TPG * 1024 + (16 * h) * 4 + g * 4);
+                const uint32_t so1 = lds32(chunk + TPG * 1024 + (16 * h + 8) * 4 + g * 4);
+                const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&so0));  // (scale, offset)
+                const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&so1));
+                acc[h][0] = fmaf(r0.x, d[h][0], fmaf(r0.y, sx_even, acc[h][0]));
+                acc[h][1] = fmaf(r0.x, d[h][1], fmaf(r0.y, sx_odd, acc[h][1]));
+                acc[h][2] = fmaf(r1.x, d[h][2], fmaf(r1.y, sx_even, acc[h][2]));
+                acc[h][3] = fmaf(r1.x, d[h][3], fmaf(r1.y, sx_odd, acc[h][3]));
             }
+            __syncwarp();  // every lane has read the slot before the next refill targets it
+            chunk += CH;
+            if (chunk >= ring_end) chunk = ring;
+            xo += uint32_t(S) * G * (XS ? 2u : 1u);
+            gsp += S * 64;
         }
-        buf ^= 1;
+        // element e = 8 lane + 4 h + i is (row 16 h + g + 8 (i / 2), vector 2 t + (i % 2)) of the strip
+        if (S == 1) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = 32 * strip + 16 * h + g + 8 * (i >> 1), v = 2 * t + (i & 1);
+                    if (row < N && v < batch) y[size_t(v) * N + row] = acc[h][i];
+                }
+        } else {
+            float* mine = red + warp * 256 + 8 * lane;
+            *reinterpret_cast<float4*>(mine) = make_float4(acc[0][0], acc[0][1], acc[0][2], acc[0][3]);
+            *reinterpret_cast<float4*>(mine + 4) = make_float4(acc[1][0], acc[1][1], acc[1][2], acc[1][3]);
+            team_barrier(team, S);
+            const float* first = red + team * S * 256;
+            for (int e = p * 32 + lane; e < 256; e += S * 32) {
+                const int el = e >> 3, h = (e >> 2) & 1, i = e & 3;
+                const int row = 32 * strip + 16 * h + (el >> 2) + 8 * (i >> 1), v = 2 * (el & 3) + (i & 1);
+                if (row < N && v < batch) {
+                    float total = 0.f;
+                    for (int k = 0; k < S; ++k) total += first[k * 256 + e];  // warp order: fixed
+                    y[size_t(v) * N + row] = total;
+                }
+            }
+            team_barrier(team, S);  // the sums have been read before the next strip overwrites them
+        }
     }
+    q4_cp_async_wait<0>();
 }
 
-// One thread per (token, tile, t, m): four consecutive weights of the row as float16 (Sec. 4.4).
-__global__ void __launch_bounds__(256) k_q4_rows(const uint32_t* __restrict__ packed, const int32_t* __restrict__ ids,
+// One thread per (token, four consecutive columns): float16 weights of the row (Sec. 4.4).
+__global__ void __launch_bounds__(256) k_q4_rows(const unsigned char* __restrict__ packed, const int32_t* __restrict__ ids,
                                                  int count, __half* __restrict__ out, int N, int K, int G) {
-    const int strips = (N + 15) / 16, KT = K / 64, groups = K / G;
-    const uint32_t* so = packed + size_t(strips) * KT * 128;
-    const size_t per_row = size_t(KT) * 16;
+    const int groups = K / G, CH = q4_chunk_bytes(G), tile_bytes = (G / 64) * 1024;
+    const size_t per_row = size_t(K / 4);
     pdl_release();
     pdl_wait();  // the ids may come from the preceding kernel
     for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < size_t(count) * per_row;
          i += size_t(gridDim.x) * blockDim.x) {
         const int tok = int(i / per_row);
-        const int rem = int(i % per_row);
-        const int m = rem & 3, t = (rem >> 2) & 3, kt = rem >> 4;
-        const int c = 64 * kt + 16 * t + 4 * m;
+        const int c = 4 * int(i % per_row);
         const int row = ids[tok];
         uint2 res = make_uint2(0u, 0u);
         if (row >= 0 && row < N) {
-            const int strip = row >> 4, g = row & 7, half = (row >> 3) & 1;
-            const uint32_t w = packed[((size_t(strip) * KT + kt) * 32 + g * 4 + t) * 4 + m] >> (8 * half);
-            const uint32_t rec = so[(size_t(strip) * groups + c / G) * 16 + (row & 15)];
+            const int strip = row >> 5, rr = row & 31, h = rr >> 4, g = rr & 7, half = (rr >> 3) & 1;
+            const int group = c / G, cg = c % G, j = cg >> 6, t = (cg >> 4) & 3, m = (cg >> 2) & 3;
+            const unsigned char* chunk = packed + (size_t(strip) * groups + group) * CH;
+            const uint32_t w = *reinterpret_cast<const uint32_t*>(chunk + j * 1024 + h * 512 + (g * 4 + t) * 16 + m * 4) >>
+                               (8 * half);
+            const uint32_t rec = *reinterpret_cast<const uint32_t*>(chunk + tile_bytes + rr * 4);
             const float2 sc = __half22float2(*reinterpret_cast<const __half2*>(&rec));
             const float n0 = float(w & 15u), n1 = float((w >> 16) & 15u);        // columns c, c + 1
             const float n2 = float((w >> 4) & 15u), n3 = float((w >> 20) & 15u);  // columns c + 2, c + 3
@@ -265,23 +362,29 @@ int device_sm_count(int* sms) {
     return cuda_status(e);
 }
 
-template <int G>
-cudaError_t launch_q4_gemv(const void* packed, const void* x, float* y, int N, int K, int batch, int sms,
-                           cudaStream_t s) {
-    const int strips = (N + 15) / 16, groups = K / G;
-    // team size: enough (strip, group-slice) units for two CTAs of 16 warps per SM
+constexpr size_t kQ4SmemLimit = 224 * 1024 / kQ4CtasPerSm - 2048;
+constexpr size_t kQ4StageLimit = 40 * 1024;  // activations up to this size are staged in shared memory
+
+template <int G, int DEPTH, bool XS>
+cudaError_t launch_q4_variant(const void* packed, const void* x, float* y, int N, int K, int batch, int sms,
+                              cudaStream_t s) {
+    const int strips = (N + 31) / 32, groups = K / G;
+    // team size: enough (strip, group-slice) units for every resident warp
     int S = 1;
-    while (S < kQ4Warps && S * 2 <= groups && size_t(strips) * S < size_t(2) * sms * kQ4Warps) S *= 2;
+    while (S < kQ4Warps && S * 2 <= groups && size_t(strips) * S < size_t(kQ4CtasPerSm) * sms * kQ4Warps) S *= 2;
     const int teams = kQ4Warps / S;
     int grid = (strips + teams - 1) / teams;
-    if (grid > 2 * sms) grid = 2 * sms;
-    const size_t smem = size_t(groups) * 64 + size_t(2) * kQ4Warps * 128 * 4;
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[G == 128]) {
-        cudaError_t e = cudaFuncSetAttribute(k_q4_gemv<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+    if (grid > kQ4CtasPerSm * sms) grid = kQ4CtasPerSm * sms;
+    const size_t smem = size_t(groups) * 64 + size_t(kQ4Warps) * 1024 + size_t(kQ4Warps) * DEPTH * q4_chunk_bytes(G) +
+                        (XS ? size_t(batch) * (size_t(K) * 2 + 16) : 0);
+    static bool attr_set = false;  // one flag per instantiation
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_q4_gemv<G, DEPTH, XS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             int(kQ4SmemLimit));
         if (e != cudaSuccess) return e;
-        attr_set[G == 128] = true;
+        attr_set = true;
     }
+    if (smem > kQ4SmemLimit) return cudaErrorInvalidValue;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -292,8 +395,16 @@ cudaError_t launch_q4_gemv(const void* packed, const void* x, float* y, int N, i
     cfg.stream = s;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_q4_gemv<G>, static_cast<const uint4*>(packed), static_cast<const __half*>(x), y,
-                              N, K, batch, S);
+    return cudaLaunchKernelEx(&cfg, k_q4_gemv<G, DEPTH, XS>, static_cast<const unsigned char*>(packed),
+                              static_cast<const __half*>(x), y, N, K, batch, S);
+}
+
+template <int G, int DEPTH>
+cudaError_t launch_q4_gemv(const void* packed, const void* x, float* y, int N, int K, int batch, int sms,
+                           cudaStream_t s) {
+    if (size_t(batch) * (size_t(K) * 2 + 16) <= kQ4StageLimit)
+        return launch_q4_variant<G, DEPTH, true>(packed, x, y, N, K, batch, sms, s);
+    return launch_q4_variant<G, DEPTH, false>(packed, x, y, N, K, batch, sms, s);
 }
 
 }  // namespace
@@ -305,8 +416,7 @@ extern "C" {
 
 size_t tetra_q4_packed_bytes(int N, int K, int G) {
     if (check_shape(N, K, G) != TETRA_OK) return 0;
-    const int strips = (N + 15) / 16;
-    return q4_weight_bytes(strips, K) + size_t(strips) * (K / G) * 16 * 4;
+    return size_t((N + 31) / 32) * (K / G) * q4_chunk_bytes(G);
 }
 
 int tetra_q4_pack(const void* q_dev, const void* scale_dev, const void* offset_dev, void* packed_dev,
@@ -334,13 +444,12 @@ int tetra_q4_gemv(const void* packed_dev, const void* x_dev, float* y_dev, int N
     if (rc != TETRA_OK) return rc;
     if (batch < 1 || batch > TETRA_Q4_MAX_BATCH) return TETRA_ERR_BATCH;
     if (!aligned(packed_dev, 16) || !aligned(x_dev, 16) || !aligned(y_dev, 4)) return TETRA_ERR_ALIGN;
-    if (size_t(K / G) * 64 + 16384 > 96 * 1024) return TETRA_ERR_SHAPE;
     int sms = 0;
     const int drc = device_sm_count(&sms);
     if (drc != TETRA_OK) return drc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    return cuda_status(G == 128 ? launch_q4_gemv<128>(packed_dev, x_dev, y_dev, N, K, batch, sms, s)
-                                : launch_q4_gemv<64>(packed_dev, x_dev, y_dev, N, K, batch, sms, s));
+    return cuda_status(G == 128 ? launch_q4_gemv<128, 3>(packed_dev, x_dev, y_dev, N, K, batch, sms, s)
+                                : launch_q4_gemv<64, 6>(packed_dev, x_dev, y_dev, N, K, batch, sms, s));
 }
 
 int tetra_q4_rows(const void* packed_dev, const int32_t* ids_dev, int count, void* out_dev, int N, int K, int G,
@@ -363,7 +472,7 @@ int tetra_q4_rows(const void* packed_dev, const int32_t* ids_dev, int count, voi
     cfg.stream = static_cast<cudaStream_t>(stream);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cuda_status(cudaLaunchKernelEx(&cfg, k_q4_rows, static_cast<const uint32_t*>(packed_dev), ids_dev, count,
+    return cuda_status(cudaLaunchKernelEx(&cfg, k_q4_rows, static_cast<const unsigned char*>(packed_dev), ids_dev, count,
                                           static_cast<__half*>(out_dev), N, K, G));
 }
 
