@@ -104,20 +104,14 @@ __device__ __forceinline__ void q4_cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
 }
 
-__device__ __forceinline__ void team_barrier(int team, int team_warps) {
-    if (team_warps == 1)
-        __syncwarp();
-    else
-        asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(team_warps * 32) : "memory");
-}
-
-// A team of S warps (S a power of two, 1..16) owns a strip of 32 rows at a time and splits its groups: warp p
-// of the team takes groups p, p + S, ...  The warp's chunks, across all its strips, form one stream that it
-// copies into a ring of DEPTH slots in shared memory with cp.async, DEPTH - 1 chunks ahead.  Per chunk: the
+// A CTA owns a contiguous range of 32-row strips (equal shares), and its 16 warps cut the CTA's chunks, in
+// memory order, into 16 equal contiguous ranges: every warp streams one contiguous piece of the matrix
+// through a ring of DEPTH slots in shared memory (cp.async, DEPTH - 1 chunks ahead).  Per chunk: the
 // accumulators of the two 16-row sub-tiles start at minus the group's sum(bias_k x_k), every 64-column tile
 // adds four MMAs per sub-tile (the activations' B fragments are shared by both), then
 //     acc += scale * D + offset * sum_group(x).
-// At the end of a strip the team's warps add their sums through shared memory (S > 1) and store.
+// A strip that lies wholly inside a warp's range is stored directly; a strip cut by a range boundary leaves
+// one piece per warp in shared memory, and after one CTA barrier the pieces are added in warp order.
 // Addresses advance by running pointers: the loop body is dequantise, multiply, scale.
 // First MMA of a group: the accumulator starts from c (minus the group's bias sums).
 __device__ __forceinline__ void mma_f16_first(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1, float c_even,
@@ -132,48 +126,46 @@ __device__ __forceinline__ void mma_f16_first(float (&d)[4], const uint32_t (&a)
 template <int G, int DEPTH, bool XS>
 __global__ void __launch_bounds__(kQ4Threads, kQ4CtasPerSm)
 k_q4_gemv(const unsigned char* __restrict__ packed, const __half* __restrict__ x, float* __restrict__ y, int N, int K,
-          int batch, int S) {
+          int batch) {
     constexpr int TPG = G / 64, CH = q4_chunk_bytes(G), PIECES = CH / 16;
     extern __shared__ __align__(16) unsigned char q4_smem[];
+    __shared__ int piece_strip[2 * kQ4Warps];
     const int groups = K / G, strips = (N + 31) / 32;
     float2* gs = reinterpret_cast<float2*>(q4_smem);                        // [groups][8]: (sum x, -sum bias x)
-    float* red = reinterpret_cast<float*>(q4_smem + size_t(groups) * 64);   // [warps][256]
+    float* pieces = reinterpret_cast<float*>(q4_smem + size_t(groups) * 64);  // [warps][2][256]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t ring = smem_u32(q4_smem + size_t(groups) * 64 + kQ4Warps * 1024) + uint32_t(warp) * (DEPTH * CH);
-    unsigned char* xs_base = q4_smem + size_t(groups) * 64 + kQ4Warps * 1024 + size_t(kQ4Warps) * DEPTH * CH;
+    constexpr int kPieceBytes = kQ4Warps * 2 * 1024;
+    const uint32_t ring = smem_u32(q4_smem + size_t(groups) * 64 + kPieceBytes) + uint32_t(warp) * (DEPTH * CH);
+    unsigned char* xs_base = q4_smem + size_t(groups) * 64 + kPieceBytes + size_t(kQ4Warps) * DEPTH * CH;
     const uint32_t xs_stride = uint32_t(K) * 2u + 16u;  // bytes per staged vector
-    const uint32_t ring_end = ring + DEPTH * CH;
     const int g = lane >> 2, t = lane & 3;
     pdl_release();
+    if (threadIdx.x < 2 * kQ4Warps) piece_strip[threadIdx.x] = -1;
 
-    const int teams = kQ4Warps / S, team = warp / S, p = warp % S;
-    const int cnt = p < groups ? (groups - p + S - 1) / S : 0;  // chunks of this warp per strip
-    const int strip0 = blockIdx.x * teams + team, strip_step = gridDim.x * teams;
-    const int my_strips = strip0 < strips ? (strips - strip0 + strip_step - 1) / strip_step : 0;
-    // fetch cursor over the warp's stream of chunks (all its strips, one after the other)
-    const unsigned char* f_src = packed + (size_t(strip0) * groups + p) * CH + lane * 16;
-    const uint32_t f_wrap_chunks = uint32_t(strip_step) * uint32_t(groups) - uint32_t(cnt > 0 ? cnt - 1 : 0) * uint32_t(S);
-    int f_left = my_strips * cnt, f_in_strip = cnt;
-    uint32_t f_dst = ring + lane * 16;
-    auto fetch = [&]() {
-        if (f_left > 0) {
+    // this CTA's strips, this warp's chunks (local index n = local strip * groups + group)
+    const int strip_begin = int(size_t(blockIdx.x) * strips / gridDim.x);
+    const int strip_end = int((size_t(blockIdx.x) + 1) * strips / gridDim.x);
+    const uint32_t cta_chunks = uint32_t(strip_end - strip_begin) * uint32_t(groups);
+    const uint32_t n_begin = uint32_t(uint64_t(warp) * cta_chunks / kQ4Warps);
+    const uint32_t n_end = uint32_t((uint64_t(warp) + 1) * cta_chunks / kQ4Warps);
+    // running addresses: f_src = next chunk to copy (this lane's 16 bytes of each 512), f_todo = chunks left to
+    // copy; slot_lane = this lane's 16 bytes in the slot being consumed; the slot consumed last is refilled
+    const unsigned char* f_src = packed + (size_t(strip_begin) * groups + n_begin) * CH + lane * 16;
+    int f_todo = int(n_end - n_begin);
+    const uint32_t ring_lane = ring + lane * 16, ring_lane_end = ring_lane + DEPTH * CH;
+    const bool tail_lane = lane < PIECES % 32;  // lanes that copy the last, partial group of 16-byte pieces
+    auto fetch_into = [&](uint32_t dst_lane) {
+        if (f_todo > 0) {
 #pragma unroll
-            for (int i = 0; i < (PIECES + 31) / 32; ++i)
-                if ((i + 1) * 32 <= PIECES || lane < PIECES - i * 32) q4_cp_async16(f_dst + i * 512, f_src + i * 512);
-            --f_left;
-            if (--f_in_strip == 0) {
-                f_in_strip = cnt;
-                f_src += size_t(f_wrap_chunks) * CH;
-            } else {
-                f_src += size_t(uint32_t(S)) * CH;
-            }
+            for (int i = 0; i < PIECES / 32; ++i) q4_cp_async16(dst_lane + i * 512, f_src + i * 512);
+            if (PIECES % 32 != 0 && tail_lane) q4_cp_async16(dst_lane + (PIECES / 32) * 512, f_src + (PIECES / 32) * 512);
+            f_src += CH;
         }
-        f_dst += CH;
-        if (f_dst >= ring_end) f_dst -= DEPTH * CH;
+        --f_todo;
         asm volatile("cp.async.commit_group;" ::: "memory");  // one group per call, empty or not
     };
 #pragma unroll
-    for (int i = 0; i < DEPTH - 1; ++i) fetch();  // the weights do not depend on the preceding kernel
+    for (int i = 0; i < DEPTH - 1; ++i) fetch_into(ring_lane + i * CH);  // the weights do not depend on the preceding kernel
 
     pdl_wait();  // x may come from the preceding kernel
     if (XS) {
@@ -182,49 +174,61 @@ k_q4_gemv(const unsigned char* __restrict__ packed, const __half* __restrict__ x
             *reinterpret_cast<uint4*>(xs_base + size_t(v) * xs_stride + size_t(c8) * 16) =
                 __ldg(reinterpret_cast<const uint4*>(x + size_t(v) * K) + c8);
         }
+        __syncthreads();
     }
-    // per (group, vector): sum of x and minus the sum of bias_k x_k, bias 1024 for k % 4 in {0, 1}, 64 for {2, 3}
-    for (int task = threadIdx.x; task < groups * 8; task += kQ4Threads) {
-        const int v = task & 7, gi = task >> 3;
-        float sx = 0.f, sb = 0.f;
+    // per (group, vector): sum of x and minus the sum of bias_k x_k, bias 1024 for k % 4 in {0, 1}, 64 for {2, 3};
+    // eight lanes per task, combined by shuffles in a fixed order
+    for (int task0 = (threadIdx.x >> 3); task0 < groups * 8; task0 += kQ4Threads / 8) {
+        const int v = task0 & 7, gi = task0 >> 3, sub = threadIdx.x & 7;
+        float lo = 0.f, hi = 0.f;  // k % 4 in {0, 1} / {2, 3}
         if (v < batch) {
-            const uint2* src = reinterpret_cast<const uint2*>(x + size_t(v) * K + size_t(gi) * G);
-            float lo = 0.f, hi = 0.f;  // k % 4 in {0, 1} / {2, 3}
-#pragma unroll 4
-            for (int i = 0; i < G / 4; ++i) {
-                const uint2 u = __ldg(src + i);
+            const uint2* src = XS ? reinterpret_cast<const uint2*>(xs_base + size_t(v) * xs_stride) + size_t(gi) * (G / 4)
+                                  : reinterpret_cast<const uint2*>(x + size_t(v) * K + size_t(gi) * G);
+#pragma unroll
+            for (int i = 0; i < G / 32; ++i) {
+                const uint2 u = XS ? src[sub + 8 * i] : __ldg(src + sub + 8 * i);
                 const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&u.x));
                 const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
                 lo += a.x + a.y;
                 hi += b.x + b.y;
             }
-            sx = lo + hi;
-            sb = -(1024.f * lo + 64.f * hi);
         }
-        gs[task] = make_float2(sx, sb);
+#pragma unroll
+        for (int o = 4; o >= 1; o >>= 1) {
+            lo += __shfl_xor_sync(0xFFFFFFFFu, lo, o);
+            hi += __shfl_xor_sync(0xFFFFFFFFu, hi, o);
+        }
+        if (sub == 0) gs[task0] = make_float2(lo + hi, -(1024.f * lo + 64.f * hi));
     }
     __syncthreads();
 
     // column g of B is vector g; columns at or beyond batch are never stored, so they may hold any vector
     const uint32_t x_vec = uint32_t(g < batch ? g : batch - 1);
-    // this lane's 16 activations of the first tile of group p: an offset in halves (global) or a shared address
-    const uint32_t x_lane = XS ? smem_u32(xs_base) + x_vec * xs_stride + (16u * t + uint32_t(p) * G) * 2u
-                               : x_vec * uint32_t(K) + 16u * t + uint32_t(p) * G;
-    const uint32_t gs_lane = smem_u32(gs) + uint32_t(p) * 64 + uint32_t(t) * 16;
-    uint32_t chunk = ring;
-    int strip = strip0;
-    for (int si = 0; si < my_strips; ++si, strip += strip_step) {
+    // this lane's 16 activations of the first tile of group 0: an offset in halves (global) or a shared address
+    const uint32_t x_lane = XS ? smem_u32(xs_base) + x_vec * xs_stride + 32u * t : x_vec * uint32_t(K) + 16u * t;
+    const uint32_t gs_lane = smem_u32(gs) + uint32_t(t) * 16;
+    uint32_t slot_lane = ring_lane;                       // slot being consumed
+    uint32_t refill_lane = ring_lane + (DEPTH - 1) * CH;  // slot consumed last (empty at the start)
+    const uint32_t so_delta = uint32_t(TPG * 1024 + g * 4) - uint32_t(lane * 16);  // slot_lane -> this lane's scale records
+    int gi = int(n_begin % uint32_t(groups));
+    int strip = strip_begin + int(n_begin / uint32_t(groups));
+    int n_pieces = 0;
+    uint32_t left = n_end - n_begin;
+    while (left > 0) {
+        // one segment: the chunks of this warp that belong to one strip
+        const int seg_first = gi;
+        const uint32_t seg_len = min(uint32_t(groups - gi), left);
+        uint32_t xo = x_lane + uint32_t(gi) * G * (XS ? 2u : 1u);
+        uint32_t gsp = gs_lane + uint32_t(gi) * 64;
         float acc[2][4];
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[h][i] = 0.f;
-        uint32_t xo = x_lane;
-        uint32_t gsp = gs_lane;
-        for (int idx = 0; idx < cnt; ++idx) {
+        for (uint32_t c = 0; c < seg_len; ++c) {
             uint32_t cs[4];  // (sum x, -sum bias x) of vectors 2 t, 2 t + 1
             q4_lds128(gsp, cs);
-            fetch();                        // refill the slot consumed last
+            fetch_into(refill_lane);
             q4_cp_async_wait<DEPTH - 1>();  // this chunk has landed
             __syncwarp();
             float d[2][4];
@@ -250,7 +254,7 @@ k_q4_gemv(const unsigned char* __restrict__ packed, const __half* __restrict__ x
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     uint32_t ww[4];
-                    q4_lds128(chunk + j * 1024 + h * 512 + lane * 16, ww);
+                    q4_lds128(slot_lane + j * 1024 + h * 512, ww);
 #pragma unroll
                     for (int m = 0; m < 4; ++m) {
                         uint32_t a[4];
@@ -268,10 +272,11 @@ k_q4_gemv(const unsigned char* __restrict__ packed, const __half* __restrict__ x
             }
             // this lane's results: rows 16 h + g (i = 0, 1) and 16 h + g + 8 (i = 2, 3), vectors 2 t + (i & 1)
             const float sx_even = __uint_as_float(cs[0]), sx_odd = __uint_as_float(cs[2]);
+            const uint32_t so_lane = slot_lane + so_delta;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const uint32_t so0 = lds32(chunk + TPG * 1024 + (16 * h) * 4 + g * 4);
-                const uint32_t so1 = lds32(chunk + TPG * 1024 + (16 * h + 8) * 4 + g * 4);
+                const uint32_t so0 = lds32(so_lane + 64 * h);
+                const uint32_t so1 = lds32(so_lane + 64 * h + 32);
                 const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&so0));  // (scale, offset)
                 const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&so1));
                 acc[h][0] = fmaf(r0.x, d[h][0], fmaf(r0.y, sx_even, acc[h][0]));
@@ -280,13 +285,16 @@ k_q4_gemv(const unsigned char* __restrict__ packed, const __half* __restrict__ x
                 acc[h][3] = fmaf(r1.x, d[h][3], fmaf(r1.y, sx_odd, acc[h][3]));
             }
             __syncwarp();  // every lane has read the slot before the next refill targets it
-            chunk += CH;
-            if (chunk >= ring_end) chunk = ring;
-            xo += uint32_t(S) * G * (XS ? 2u : 1u);
-            gsp += S * 64;
+            refill_lane = slot_lane;
+            slot_lane += CH;
+            if (slot_lane == ring_lane_end) slot_lane = ring_lane;
+            xo += G * (XS ? 2u : 1u);
+            gsp += 64;
         }
+        left -= seg_len;
+        gi += int(seg_len);
         // element e = 8 lane + 4 h + i is (row 16 h + g + 8 (i / 2), vector 2 t + (i % 2)) of the strip
-        if (S == 1) {
+        if (seg_first == 0 && gi == groups) {  // the whole strip was this warp's
 #pragma unroll
             for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -294,25 +302,37 @@ k_q4_gemv(const unsigned char* __restrict__ packed, const __half* __restrict__ x
                     const int row = 32 * strip + 16 * h + g + 8 * (i >> 1), v = 2 * t + (i & 1);
                     if (row < N && v < batch) y[size_t(v) * N + row] = acc[h][i];
                 }
-        } else {
-            float* mine = red + warp * 256 + 8 * lane;
+        } else {  // a strip shared with a neighbouring warp: leave a piece
+            float* mine = pieces + (2 * warp + n_pieces) * 256 + 8 * lane;
             *reinterpret_cast<float4*>(mine) = make_float4(acc[0][0], acc[0][1], acc[0][2], acc[0][3]);
             *reinterpret_cast<float4*>(mine + 4) = make_float4(acc[1][0], acc[1][1], acc[1][2], acc[1][3]);
-            team_barrier(team, S);
-            const float* first = red + team * S * 256;
-            for (int e = p * 32 + lane; e < 256; e += S * 32) {
-                const int el = e >> 3, h = (e >> 2) & 1, i = e & 3;
-                const int row = 32 * strip + 16 * h + (el >> 2) + 8 * (i >> 1), v = 2 * (el & 3) + (i & 1);
-                if (row < N && v < batch) {
-                    float total = 0.f;
-                    for (int k = 0; k < S; ++k) total += first[k * 256 + e];  // warp order: fixed
-                    y[size_t(v) * N + row] = total;
-                }
-            }
-            team_barrier(team, S);  // the sums have been read before the next strip overwrites them
+            if (lane == 0) piece_strip[2 * warp + n_pieces] = strip;
+            ++n_pieces;
+        }
+        if (gi == groups) {
+            gi = 0;
+            ++strip;
         }
     }
     q4_cp_async_wait<0>();
+    __syncthreads();
+    // pieces in (warp, first/second) order are in memory order: the pieces of a strip are consecutive
+    if (threadIdx.x < 256) {
+        const int e = threadIdx.x, el = e >> 3, h = (e >> 2) & 1, i = e & 3;
+        const int r_in = 16 * h + (el >> 2) + 8 * (i >> 1), v = 2 * (el & 3) + (i & 1);
+        int cur = -1;
+        float total = 0.f;
+        for (int pc = 0; pc <= 2 * kQ4Warps; ++pc) {
+            const int sidx = pc < 2 * kQ4Warps ? piece_strip[pc] : -2;
+            if (sidx == -1) continue;
+            if (sidx != cur) {
+                if (cur >= 0 && 32 * cur + r_in < N && v < batch) y[size_t(v) * N + 32 * cur + r_in] = total;
+                cur = sidx;
+                total = 0.f;
+            }
+            if (sidx >= 0) total += pieces[pc * 256 + e];
+        }
+    }
 }
 
 // One thread per (token, four consecutive columns): float16 weights of the row (Sec. 4.4).
@@ -369,13 +389,8 @@ template <int G, int DEPTH, bool XS>
 cudaError_t launch_q4_variant(const void* packed, const void* x, float* y, int N, int K, int batch, int sms,
                               cudaStream_t s) {
     const int strips = (N + 31) / 32, groups = K / G;
-    // team size: enough (strip, group-slice) units for every resident warp
-    int S = 1;
-    while (S < kQ4Warps && S * 2 <= groups && size_t(strips) * S < size_t(kQ4CtasPerSm) * sms * kQ4Warps) S *= 2;
-    const int teams = kQ4Warps / S;
-    int grid = (strips + teams - 1) / teams;
-    if (grid > kQ4CtasPerSm * sms) grid = kQ4CtasPerSm * sms;
-    const size_t smem = size_t(groups) * 64 + size_t(kQ4Warps) * 1024 + size_t(kQ4Warps) * DEPTH * q4_chunk_bytes(G) +
+    int grid = strips < kQ4CtasPerSm * sms ? strips : kQ4CtasPerSm * sms;
+    const size_t smem = size_t(groups) * 64 + size_t(kQ4Warps) * 2048 + size_t(kQ4Warps) * DEPTH * q4_chunk_bytes(G) +
                         (XS ? size_t(batch) * (size_t(K) * 2 + 16) : 0);
     static bool attr_set = false;  // one flag per instantiation
     if (!attr_set) {
@@ -396,7 +411,7 @@ cudaError_t launch_q4_variant(const void* packed, const void* x, float* y, int N
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, k_q4_gemv<G, DEPTH, XS>, static_cast<const unsigned char*>(packed),
-                              static_cast<const __half*>(x), y, N, K, batch, S);
+                              static_cast<const __half*>(x), y, N, K, batch);
 }
 
 template <int G, int DEPTH>
