@@ -176,6 +176,9 @@ def main():
     ap.add_argument("--batched-only", type=int, default=0, metavar="VECTORS",
                     help="profiling runs: two rounds of tetra_gemv_batched over 12 copies of the 4096 x 12288 "
                          "matrix with this many vectors, nothing else, no JSON line")
+    ap.add_argument("--q4-only", default="", metavar="N,K,G,BATCH",
+                    help="profiling runs: three tetra_q4_gemv launches on one synthetic matrix, nothing else, "
+                         "no JSON line")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -204,6 +207,20 @@ def main():
     elif not os.path.exists(tbuild.LIB) and not os.environ.get("TETRA_LIB"):
         tbuild.build()
 
+    if args.q4_only:
+        from paper_2609_35465_b200 import synth, tetra
+        qN, qK, qG, qB = (int(v) for v in args.q4_only.split(","))
+        rows_src = min(qN, 4096)
+        qn = torch.from_numpy(synth.q4_nibbles(args.seed + 17, qN, rows_src, qK)).cuda()
+        qn = qn.repeat((qN + rows_src - 1) // rows_src, 1)[:qN].contiguous()
+        sc, of = synth.q4_scales_offsets(args.seed + 17, qN, qN, qK // qG)
+        pk = tetra.tetra_q4_pack(qn, torch.from_numpy(sc).cuda(), torch.from_numpy(of).cuda(), qN, qK, qG)
+        xq = torch.from_numpy(synth.activations(args.seed + 17, 1, qK, qB)).cuda()
+        yq = torch.empty((qB, qN), dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            tetra.tetra_q4_gemv(pk, xq, yq, qN, qK, qG, qB)
+        torch.cuda.synchronize()
+        return
     if args.batched_only:
         from paper_2609_35465_b200 import synth, tetra
         m = shapes.CONFIG4
@@ -365,6 +382,44 @@ def main():
                                  "weights_x_vectors_per_s": m.N * m.K * batch / us["batched"] * 1e6}
         out["batch_sweep_4096x12288"] = sweep
         del one, ws
+
+        # 4-bit group-quantised matrices (the served model's other weight format): the int4 projection shapes
+        # of this model (groups of 128) and the output head (151,936 rows, groups of 64), batch 1, CUDA graph
+        # over distinct copies (more than L2 together), after half a second of the same work
+        q4 = {}
+        kv_dim, q_dim = model.kv_heads * model.head_dim, model.q_heads * model.head_dim
+        q4_shapes = [("v_proj", kv_dim, model.hidden, 128, 48), ("o_proj", model.hidden, q_dim, 128, 24),
+                     ("down_proj", model.hidden, model.intermediate, 128, 12),
+                     ("head", 151936, model.hidden, 64, 2)]
+        for name, qN, qK, qG, copies in q4_shapes:
+            rows_src = min(qN, 4096)  # the head repeats a 4096-row pattern of nibbles: timing only
+            qn = torch.from_numpy(synth.q4_nibbles(args.seed + 17, qN, rows_src, qK)).cuda()
+            qn = qn.repeat((qN + rows_src - 1) // rows_src, 1)[:qN].contiguous()
+            sc, of = synth.q4_scales_offsets(args.seed + 17, qN, qN, qK // qG)
+            sc, of = torch.from_numpy(sc).cuda(), torch.from_numpy(of).cuda()
+            packs = [tetra.tetra_q4_pack(qn, sc, of, qN, qK, qG) for _ in range(copies)]
+            xq = torch.from_numpy(synth.activations(args.seed + 17, 1, qK, 1)).cuda()
+            yq = torch.empty((1, qN), dtype=torch.float32, device="cuda")
+
+            def run_q4(stream=None):
+                for pk in packs:
+                    tetra.tetra_q4_gemv(pk, xq, yq, qN, qK, qG, 1, stream=stream)
+            run_q4()
+            gg = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gg, stream=torch.cuda.Stream()):
+                run_q4(stream=torch.cuda.current_stream())
+            t_end = time.time() + 0.5
+            while time.time() < t_end:
+                gg.replay()
+                torch.cuda.synchronize()
+            us = timed(torch, gg.replay, 20, 3, stream) * 1e3 / copies
+            nbytes = packs[0].numel() + 2 * qK + 4 * qN
+            q4[name] = {"N": qN, "K": qK, "group": qG, "us": us, "algorithmic_bytes": nbytes, "GBps": nbytes / us / 1e3,
+                        "frac_of_measured_peak": nbytes / us / 1e3 / peak_now, "roofline_us": nbytes / peak_now / 1e3,
+                        "bits_per_weight": 8.0 * packs[0].numel() / (qN * qK)}
+            del packs, gg, qn, sc, of
+            torch.cuda.empty_cache()
+        out["q4_gemv"] = q4
 
         # the other two model sizes, planned-list pass (same kernels; a few repetitions)
         others = {}

@@ -88,6 +88,16 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], u
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// (a, a) * (b0, b1) + (c0, c1) in one instruction (fma.rn.f32x2).
+__device__ __forceinline__ void fma2(float a, float b0, float b1, float& c0, float& c1) {
+    uint64_t aa, bb, cc;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(aa) : "f"(a));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(bb) : "f"(b0), "f"(b1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(cc) : "f"(c0), "f"(c1));
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(cc) : "l"(aa), "l"(bb));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(c0), "=f"(c1) : "l"(cc));
+}
+
 __device__ __forceinline__ uint32_t lop_and_or(uint32_t a, uint32_t mask, uint32_t magic) {
     uint32_t r;
     asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(magic));  // (a & mask) | magic
@@ -279,10 +289,10 @@ k_q4_gemv(const unsigned char* __restrict__ packed, const __half* __restrict__ x
                 const uint32_t so1 = lds32(so_lane + 64 * h + 32);
                 const float2 r0 = __half22float2(*reinterpret_cast<const __half2*>(&so0));  // (scale, offset)
                 const float2 r1 = __half22float2(*reinterpret_cast<const __half2*>(&so1));
-                acc[h][0] = fmaf(r0.x, d[h][0], fmaf(r0.y, sx_even, acc[h][0]));
-                acc[h][1] = fmaf(r0.x, d[h][1], fmaf(r0.y, sx_odd, acc[h][1]));
-                acc[h][2] = fmaf(r1.x, d[h][2], fmaf(r1.y, sx_even, acc[h][2]));
-                acc[h][3] = fmaf(r1.x, d[h][3], fmaf(r1.y, sx_odd, acc[h][3]));
+                fma2(r0.y, sx_even, sx_odd, acc[h][0], acc[h][1]);  // offset * sum(x), vectors 2 t and 2 t + 1
+                fma2(r0.x, d[h][0], d[h][1], acc[h][0], acc[h][1]);  // scale * (sum q x)
+                fma2(r1.y, sx_even, sx_odd, acc[h][2], acc[h][3]);
+                fma2(r1.x, d[h][2], d[h][3], acc[h][2], acc[h][3]);
             }
             __syncwarp();  // every lane has read the slot before the next refill targets it
             refill_lane = slot_lane;
