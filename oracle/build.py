@@ -15,16 +15,23 @@ Q4_HDR = os.path.join(HERE, "q4_oracle.h")
 Q4_LIB = os.path.join(HERE, "libq4_oracle.so")
 
 
-def _build_one(lib: str, src: str, hdr: str, force: bool, extra=()) -> str:
+ENC_SRC = os.path.join(HERE, "tetra_encode_oracle.c")
+ENC_HDR = os.path.join(HERE, "tetra_encode_oracle.h")
+ENC_LIB = os.path.join(HERE, "libtetra_encode_oracle.so")
+
+
+def _build_one(lib: str, src, hdr, force: bool, extra=()) -> str:
+    srcs = [src] if isinstance(src, str) else list(src)
+    hdrs = [hdr] if isinstance(hdr, str) else list(hdr)
     stale = (
         force
         or not os.path.exists(lib)
-        or os.path.getmtime(lib) < max(os.path.getmtime(src), os.path.getmtime(hdr))
+        or os.path.getmtime(lib) < max(os.path.getmtime(f) for f in srcs + hdrs)
     )
     if stale:
         tmp = lib + ".tmp.%d" % os.getpid()
         cmd = ["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", *extra, "-fopenmp", "-shared", "-fPIC",
-               "-o", tmp, src, "-lm"]
+               "-o", tmp, *srcs, "-lm"]
         subprocess.run(cmd, check=True, cwd=HERE)
         os.replace(tmp, lib)
     return lib
@@ -41,6 +48,12 @@ def build_q4(force: bool = False) -> str:
     return _build_one(Q4_LIB, Q4_SRC, Q4_HDR, force, extra=("-ffp-contract=off",))
 
 
+def build_encode(force: bool = False) -> str:
+    """Build the encoder-search oracle (it calls the Tetra oracle's decoder, so both sources go in)."""
+    return _build_one(ENC_LIB, [SRC, ENC_SRC], [HDR, ENC_HDR], force)
+
+
 if __name__ == "__main__":
     print(build(force=True))
     print(build_q4(force=True))
+    print(build_encode(force=True))
