@@ -164,6 +164,19 @@ int tetra_gemv_batched(const void *codes, const float *row_scales, const void *t
                        const void *x, float *y, int N, int K, int batch, const void *tail,
                        void *workspace_dev, size_t workspace_bytes, void *stream);
 
+/* Encoder search (Sec. 3.1, Eq. (2)).  For each block of 24 float32 weights
+ * (w_dev: [nblocks][24]) finds the point of the format's codebook whose
+ * direction is closest to the block -- the exact maximum of
+ * <w, y> / (|w| |y|) over all 2^47 indices (the paper's own search is not
+ * exhaustive; the objective and the codebook are the paper's) -- and the
+ * gain bit g that minimises |w - y/|y| gain[g] sigma|^2, with gain[] from the
+ * table and sigma = sigma_dev[block] (NULL: 1).  codes_dev receives the words in
+ * file order, six bytes per block; cosine_dev (NULL allowed) the attained
+ * cosine.  A zero block gives the all-zero word and cosine 0.  Rotation, the
+ * error-feedback loop and the choice of sigma (Sec. 3.1, 4.2) are the caller's. */
+int tetra_encode_blocks(const float *w_dev, const float *sigma_dev, const void *table_dev,
+                        void *codes_dev, float *cosine_dev, size_t nblocks, void *stream);
+
 /* The design the paper describes for its own GPU (Sec. 5.1: a warp per output
  * row, a lane per block, six table loads per block), kept as a comparison arm
  * and a cross-check.  codes: file-order words, row_stride bytes per row

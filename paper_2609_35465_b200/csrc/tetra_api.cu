@@ -205,6 +205,17 @@ int tetra_gemv_batched(const void* codes, const float* row_scales, const void* t
                                            workspace_dev, as_stream(stream)));
 }
 
+int tetra_encode_blocks(const float* w_dev, const float* sigma_dev, const void* table_dev, void* codes_dev,
+                        float* cosine_dev, size_t nblocks, void* stream) {
+    if (nblocks == 0) return TETRA_OK;
+    if (!w_dev || !table_dev || !codes_dev) return TETRA_ERR_NULL;
+    if (!aligned(w_dev, 4) || !aligned(table_dev, 16) || (sigma_dev && !aligned(sigma_dev, 4)) ||
+        (cosine_dev && !aligned(cosine_dev, 4)))
+        return TETRA_ERR_ALIGN;
+    return cuda_status(launch_encode(w_dev, sigma_dev, table_dev, static_cast<unsigned char*>(codes_dev), cosine_dev,
+                                     nblocks, as_stream(stream)));
+}
+
 int tetra_gemv_paper_design(const void* codes, size_t row_stride, const float* row_scales, const void* table,
                             const void* x, float* y, int N, int K, int batch, const void* tail, void* stream) {
     if (!codes || !row_scales || !table || !x || !y) return TETRA_ERR_NULL;

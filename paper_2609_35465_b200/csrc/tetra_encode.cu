@@ -1,0 +1,429 @@
+// Encoder search (Sec. 3.1, Eq. (2)): for a block of 24 weights, the point of the format's codebook whose
+// direction is closest to the block, and the gain bit.
+//
+// The paper's own search is not exhaustive and runs on a CPU; this kernel computes the exact optimum of the
+// same objective,  max <w, y> / (|w| |y|)  over all 2^47 indices, by using what the format's structure gives:
+//   * a section's coordinates depend on (parity p, pattern byte c, rank row) only, the pattern bytes of all
+//     three sections are the 128 even-weight bytes, and for fixed (p, c, class) the section's squared norm is
+//     16 k + r with r fixed by (p, weight of c, class) and k = 0..9: per section, byte and class only ten best
+//     correlations matter (one per k);
+//   * the sections are tied by the trellis path, by the parity and by Eq. (3) (r3 = p ^ r ^ delta): they are
+//     joined state by state with the summed norm and the class parity as extra state.
+// One CTA of 384 threads works on one block at a time: three groups of 128 threads, one per section, thread =
+// pattern byte.  For every batch of 64 rank rows a group first tabulates, per row, the partial correlations and
+// norms of the 16 patterns of each half of the byte (so a (row, byte) candidate costs two shared loads and two
+// additions), then every thread scans the batch for its own byte and keeps the best correlation per (class,
+// k) in a private column of shared memory (no atomics).  The join runs on the same CTA; the rows that attain
+// the winning entries are found by a second scan of three lists.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "../../include/tetra.h"
+#include "tetra_device.cuh"
+#include "tetra_launch.h"
+#include "tetra_tables.h"
+
+namespace tetra {
+namespace {
+
+constexpr int kEncThreads = 384;
+constexpr int kEncBatch = 64;       // rank rows per batch
+constexpr int kEncStride = 65;      // row-table entries are 65 rows apart (bank spread)
+constexpr float kNeg = -1.0e30f;
+constexpr float kNegTest = -1.0e29f;
+
+struct EncShared {
+    uint32_t rows[4096];
+    uint16_t branches[1024];
+    uint8_t prefixes[128];
+    uint8_t suffixes[128];
+    uint16_t incoming[64][16];                 // per state after the branch: s8 | b2 << 6
+    int incoming_count[64];
+    float A[3][8][4][8];                       // w_j * value(o, rank)
+    uint2 rowtab[3][32 * kEncStride];          // (partial correlation, partial norm): entry (half * 16 + pattern), row
+    float T[3][20][128];                       // best correlation per (class * 10 + k), byte
+    float F1[64][2][20];                       // after section 1: state, class, norm / 8
+    float H[39][128];                          // after section 2: norm / 8, (state after the branch) * 2 + class parity
+    uint32_t Hback[39][128];
+    float red_val[kEncThreads / 32];
+    uint32_t red_arg[kEncThreads / 32];
+    float w[24];
+    // best so far
+    float best_val, best_corr;
+    int best_norm;
+    uint32_t best_path;                        // s8 | b1 << 6 | b2 << 7 | b3 << 11 | p << 12 | r << 13
+    int best_field[3];
+    int found_field[3];
+};
+
+__device__ __forceinline__ int even_byte(int ci) {  // the 128 even-weight bytes, by index
+    const int h = ci >> 3, li = ci & 7;
+    return (h << 4) | (li << 1) | ((__popc(li) ^ __popc(h)) & 1);
+}
+__device__ __forceinline__ int even_index(int byte) { return ((byte >> 4) << 3) | ((byte & 15) >> 1); }
+// squared norm of a section = 16 k + residue
+__device__ __forceinline__ int norm_residue(int p, int cls, int byte) { return p ? (cls ? 0 : 8) : ((4 * __popc(byte)) & 15); }
+
+__device__ __forceinline__ void group_barrier(int group) {
+    asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
+}
+
+// Rows of a section's list for a class: sections 0 and 2 read all 2048 rows of the class, the middle section
+// the first 1240 (class 0) or 808 (class 1) of them (Sec. 3.3).
+__device__ __forceinline__ int list_length(int section, int cls) {
+    return section == 1 ? (cls ? 2048 - kMiddleClass0 : kMiddleClass0) : 2048;
+}
+
+// Largest value over the CTA with its argument; ties go to the smaller argument.  Everyone gets the result.
+__device__ void cta_argmax(EncShared& S, float& val, uint32_t& arg) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        const float v2 = __shfl_xor_sync(0xFFFFFFFFu, val, o);
+        const uint32_t a2 = __shfl_xor_sync(0xFFFFFFFFu, arg, o);
+        if (v2 > val || (v2 == val && a2 < arg)) {
+            val = v2;
+            arg = a2;
+        }
+    }
+    __syncthreads();
+    if (lane == 0) {
+        S.red_val[warp] = val;
+        S.red_arg[warp] = arg;
+    }
+    __syncthreads();
+    val = S.red_val[0];
+    arg = S.red_arg[0];
+    for (int k = 1; k < kEncThreads / 32; ++k) {
+        const float v2 = S.red_val[k];
+        const uint32_t a2 = S.red_arg[k];
+        if (v2 > val || (v2 == val && a2 < arg)) {
+            val = v2;
+            arg = a2;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kEncThreads, 1)
+k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const DeviceTables* __restrict__ tab,
+         unsigned char* __restrict__ codes, float* __restrict__ cosine, size_t nblocks) {
+    extern __shared__ __align__(16) unsigned char enc_smem[];
+    EncShared& S = *reinterpret_cast<EncShared*>(enc_smem);
+    const int tid = threadIdx.x;
+    const int sg = tid >> 7, ct = tid & 127;  // section group, pattern-byte index
+    // --- tables, once per CTA ---
+    for (int i = tid; i < 4096; i += kEncThreads) S.rows[i] = tab->paper.rows[i];
+    for (int i = tid; i < 1024; i += kEncThreads) S.branches[i] = tab->paper.branches[i];
+    if (tid < 128) {
+        S.prefixes[tid] = tab->paper.prefixes[tid];
+        S.suffixes[tid] = tab->paper.suffixes[tid];
+    }
+    if (tid < 64) S.incoming_count[tid] = 0;
+    __syncthreads();
+    for (int i = tid; i < 1024; i += kEncThreads) {  // order within a state's list does not matter for the maximum,
+        const int s16 = S.branches[i] >> 8;          // but it decides ties: sort below
+        const int slot = atomicAdd(&S.incoming_count[s16], 1);
+        if (slot < 16) S.incoming[s16][slot] = uint16_t(i);  // i = 16 s8 + b2
+    }
+    __syncthreads();
+    if (tid < 64) {  // insertion sort of 16 entries: the same order in every CTA and run
+        for (int a = 1; a < 16; ++a) {
+            const uint16_t v = S.incoming[tid][a];
+            int b = a - 1;
+            while (b >= 0 && S.incoming[tid][b] > v) {
+                S.incoming[tid][b + 1] = S.incoming[tid][b];
+                --b;
+            }
+            S.incoming[tid][b + 1] = v;
+        }
+    }
+    const float gain0 = tab->gain[0], gain1 = tab->gain[1];
+    const int my_byte = even_byte(ct);
+    const int my_lo = my_byte & 15, my_hi = my_byte >> 4;
+    __syncthreads();
+
+    for (size_t block = blockIdx.x; block < nblocks; block += gridDim.x) {
+        if (tid < 24) S.w[tid] = w[block * 24 + tid];
+        if (tid == 0) {
+            S.best_val = kNeg;
+            S.best_corr = 0.f;
+            S.best_norm = 0;
+            S.best_path = 0;
+            S.best_field[0] = S.best_field[1] = S.best_field[2] = 0;
+        }
+        __syncthreads();
+        for (int i = tid; i < 3 * 8 * 4 * 8; i += kEncThreads) {
+            const int rho = i & 7, o = (i >> 3) & 3, j = (i >> 5) & 7, s = i >> 8;
+            S.A[s][j][o][rho] = S.w[8 * s + j] * float(rank_value(o, rho));
+        }
+        float wn2 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 24; ++j) wn2 = fmaf(S.w[j], S.w[j], wn2);
+        __syncthreads();
+        if (wn2 == 0.f) {  // a zero block encodes as the all-zero word
+            if (tid < 6) codes[block * 6 + tid] = 0;
+            if (tid == 0 && cosine) cosine[block] = 0.f;
+            continue;
+        }
+
+        for (int p = 0; p < 2; ++p) {
+            // ---------------- section tables ----------------
+            for (int i = ct; i < 20 * 128; i += 128) (&S.T[sg][0][0])[i] = kNeg;
+            group_barrier(sg);
+            for (int cls = 0; cls < 2; ++cls) {
+                const int len = list_length(sg, cls), base = 2048 * cls;
+                for (int b0 = 0; b0 < len; b0 += kEncBatch) {
+                    const int nb = min(kEncBatch, len - b0);
+                    if (ct < nb) {  // tabulate one row: 16 patterns of each half of the byte
+                        const uint32_t rw = S.rows[base + b0 + ct];
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            float P[16];
+                            int Nn[16];
+                            P[0] = 0.f;
+                            Nn[0] = 0;
+                            float d[4];
+                            int dn[4];
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj) {
+                                const int j = 4 * half + jj, rho = (rw >> (4 * j)) & 7;
+                                const float a0 = S.A[sg][j][p][rho], a1 = S.A[sg][j][p + 2][rho];
+                                const int v0 = rank_value(p, rho), v1 = rank_value(p + 2, rho);
+                                P[0] += a0;
+                                Nn[0] += v0 * v0;
+                                d[jj] = a1 - a0;
+                                dn[jj] = v1 * v1 - v0 * v0;
+                            }
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+                                for (int m = 0; m < (1 << jj); ++m) {
+                                    P[m | (1 << jj)] = P[m] + d[jj];
+                                    Nn[m | (1 << jj)] = Nn[m] + dn[jj];
+                                }
+#pragma unroll
+                            for (int m = 0; m < 16; ++m)
+                                S.rowtab[sg][(half * 16 + m) * kEncStride + ct] = make_uint2(__float_as_uint(P[m]), uint32_t(Nn[m]));
+                        }
+                    }
+                    group_barrier(sg);
+                    const uint2* lo_tab = &S.rowtab[sg][my_lo * kEncStride];
+                    const uint2* hi_tab = &S.rowtab[sg][(16 + my_hi) * kEncStride];
+                    float* my_t = &S.T[sg][cls * 10][ct];
+#pragma unroll 4
+                    for (int r = 0; r < nb; ++r) {
+                        const uint2 lo = lo_tab[r], hi = hi_tab[r];
+                        const float corr = __uint_as_float(lo.x) + __uint_as_float(hi.x);
+                        const int k = int(lo.y + hi.y) >> 4;
+                        float* cell = my_t + k * 128;
+                        *cell = fmaxf(*cell, corr);
+                    }
+                    group_barrier(sg);
+                }
+            }
+            __syncthreads();
+
+            // ---------------- join: first cut ----------------
+            for (int e = tid; e < 64 * 2 * 20; e += kEncThreads) {
+                const int n8 = e % 20, cls = (e / 20) & 1, s8 = e / 40;
+                float best = kNeg;
+#pragma unroll
+                for (int b1 = 0; b1 < 2; ++b1) {
+                    const int byte = S.prefixes[2 * s8 + b1];
+                    const int rem = 8 * n8 - norm_residue(p, cls, byte);
+                    if (rem >= 0 && (rem & 15) == 0 && (rem >> 4) < 10) best = fmaxf(best, S.T[0][cls * 10 + (rem >> 4)][even_index(byte)]);
+                }
+                S.F1[s8][cls][n8] = best;
+            }
+            for (int e = tid; e < 39 * 128; e += kEncThreads) (&S.H[0][0])[e] = kNeg;
+            __syncthreads();
+            // ---------------- second cut ----------------
+            if (tid < 128) {
+                const int s16 = tid >> 1, par = tid & 1;
+                for (int in = 0; in < 16; ++in) {
+                    const int sb = S.incoming[s16][in], s8 = sb >> 4, b2 = sb & 15;
+                    const int byte2 = S.branches[sb] & 0xFF, ci2 = even_index(byte2);
+                    for (int cls1 = 0; cls1 < 2; ++cls1) {
+                        const int cls2 = par ^ cls1, res2 = norm_residue(p, cls2, byte2) >> 3;
+                        for (int n8 = 0; n8 < 20; ++n8) {
+                            const float a = S.F1[s8][cls1][n8];
+                            if (a < kNegTest) continue;
+#pragma unroll
+                            for (int k2 = 0; k2 < 10; ++k2) {
+                                const float b = S.T[1][cls2 * 10 + k2][ci2];
+                                const int q = n8 + 2 * k2 + res2;
+                                if (b > kNegTest && a + b > S.H[q][tid]) {
+                                    S.H[q][tid] = a + b;
+                                    S.Hback[q][tid] = uint32_t(s8) | (uint32_t(b2) << 6) | (uint32_t(cls1) << 10) |
+                                                      (uint32_t(n8) << 11) | (uint32_t(k2) << 16);
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+            // ---------------- last section and the objective ----------------
+            float val = kNeg;
+            uint32_t arg = 0xFFFFFFFFu;
+            if (tid < 256) {
+                const int s16 = tid >> 2, b3 = (tid >> 1) & 1, par = tid & 1;
+                const int byte3 = S.suffixes[2 * s16 + b3], ci3 = even_index(byte3);
+                const int cls3 = p ^ par, res3 = norm_residue(p, cls3, byte3);
+                for (int q = 0; q < 39; ++q) {
+                    const float a = S.H[q][s16 * 2 + par];
+                    if (a < kNegTest) continue;
+#pragma unroll
+                    for (int k3 = 0; k3 < 10; ++k3) {
+                        const float b = S.T[2][cls3 * 10 + k3][ci3];
+                        const int n = 8 * q + 16 * k3 + res3;
+                        if (b > kNegTest && n > 0) {
+                            const float v = (a + b) / sqrtf(float(n));
+                            const uint32_t code = (uint32_t(tid) << 16) | (uint32_t(q) << 8) | uint32_t(k3);
+                            if (v > val || (v == val && code < arg)) {
+                                val = v;
+                                arg = code;
+                            }
+                        }
+                    }
+                }
+            }
+            cta_argmax(S, val, arg);
+            if (val > S.best_val) {  // uniform: resolve the path and the rows while this parity's tables are alive
+                const int wt = int(arg >> 16), q = int(arg >> 8) & 0xFF, k3 = int(arg & 0xFF);
+                const int s16 = wt >> 2, b3 = (wt >> 1) & 1, par = wt & 1;
+                const uint32_t back = S.Hback[q][s16 * 2 + par];
+                const int s8 = back & 63, b2 = (back >> 6) & 15, cls1 = (back >> 10) & 1, n8 = (back >> 11) & 31,
+                          k2 = (back >> 16) & 15;
+                const int cls2 = par ^ cls1, cls3 = p ^ par;
+                // the prefix that attains F1
+                int b1 = 0, k1 = 0;
+                {
+                    float bestv = kNeg;
+                    for (int bb = 0; bb < 2; ++bb) {
+                        const int byte = S.prefixes[2 * s8 + bb];
+                        const int rem = 8 * n8 - norm_residue(p, cls1, byte);
+                        if (rem >= 0 && (rem & 15) == 0 && (rem >> 4) < 10) {
+                            const float v = S.T[0][cls1 * 10 + (rem >> 4)][even_index(byte)];
+                            if (v > bestv) {
+                                bestv = v;
+                                b1 = bb;
+                                k1 = rem >> 4;
+                            }
+                        }
+                    }
+                }
+                const int bytes[3] = {S.prefixes[2 * s8 + b1], S.branches[16 * s8 + b2] & 0xFF, S.suffixes[2 * s16 + b3]};
+                const int clss[3] = {cls1, cls2, cls3};
+                const int ks[3] = {k1, k2, k3};
+                // second scan: group sg looks for the row of section sg (largest correlation at that byte, class, k)
+                {
+                    const int byte = bytes[sg], cls = clss[sg], kk = ks[sg];
+                    const int len = list_length(sg, cls), base = 2048 * cls;
+                    float rv = kNeg;
+                    uint32_t ra = 0xFFFFFFFFu;
+                    for (int i = ct; i < len; i += 128) {
+                        const uint32_t rw = S.rows[base + i];
+                        float corr = 0.f;
+                        int nn = 0;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const int rho = (rw >> (4 * j)) & 7, o = p + 2 * ((byte >> j) & 1);
+                            corr += S.A[sg][j][o][rho];
+                            const int v = rank_value(o, rho);
+                            nn += v * v;
+                        }
+                        if ((nn >> 4) == kk && (corr > rv || (corr == rv && uint32_t(i) < ra))) {
+                            rv = corr;
+                            ra = uint32_t(i);
+                        }
+                    }
+                    // reduce within the group of 128 threads (four warps)
+#pragma unroll
+                    for (int o = 16; o >= 1; o >>= 1) {
+                        const float v2 = __shfl_xor_sync(0xFFFFFFFFu, rv, o);
+                        const uint32_t a2 = __shfl_xor_sync(0xFFFFFFFFu, ra, o);
+                        if (v2 > rv || (v2 == rv && a2 < ra)) {
+                            rv = v2;
+                            ra = a2;
+                        }
+                    }
+                    __syncthreads();
+                    if ((tid & 31) == 0) {
+                        S.red_val[tid >> 5] = rv;
+                        S.red_arg[tid >> 5] = ra;
+                    }
+                    __syncthreads();
+                    if (ct == 0) {
+                        float bv = S.red_val[4 * sg];
+                        uint32_t ba = S.red_arg[4 * sg];
+                        for (int k = 1; k < 4; ++k) {
+                            const float v2 = S.red_val[4 * sg + k];
+                            const uint32_t a2 = S.red_arg[4 * sg + k];
+                            if (v2 > bv || (v2 == bv && a2 < ba)) {
+                                bv = v2;
+                                ba = a2;
+                            }
+                        }
+                        S.found_field[sg] = ba == 0xFFFFFFFFu ? 0 : int(ba);
+                    }
+                    __syncthreads();
+                }
+                if (tid == 0) {
+                    const int n_total = 8 * q + 16 * k3 + norm_residue(p, cls3, bytes[2]);
+                    S.best_val = val;
+                    S.best_norm = n_total;
+                    S.best_corr = val * sqrtf(float(n_total));
+                    S.best_path = uint32_t(s8) | (uint32_t(b1) << 6) | (uint32_t(b2) << 7) | (uint32_t(b3) << 11) |
+                                  (uint32_t(p) << 12) | (uint32_t(cls1) << 13);
+                    S.best_field[0] = S.found_field[0];
+                    S.best_field[1] = cls2 ? kMiddleClass0 + S.found_field[1] : S.found_field[1];
+                    S.best_field[2] = S.found_field[2];
+                }
+            }
+            __syncthreads();
+        }
+
+        if (tid == 0) {
+            const uint32_t path = S.best_path;
+            const float sg_ = sigma ? sigma[block] : 1.f;
+            // gain bit: argmin_g (gain sigma)^2 - 2 gain sigma <w, y> / |y|
+            const float c = S.best_val;
+            const float e0 = gain0 * sg_ * (gain0 * sg_ - 2.f * c), e1 = gain1 * sg_ * (gain1 * sg_ - 2.f * c);
+            const uint64_t gbit = e1 < e0 ? 1u : 0u;
+            const uint64_t word = uint64_t(S.best_field[0]) | (uint64_t(S.best_field[1]) << 11) |
+                                  (uint64_t(S.best_field[2]) << 22) | (uint64_t(path & 63u) << 33) |
+                                  (uint64_t((path >> 6) & 1u) << 39) | (uint64_t((path >> 7) & 15u) << 40) |
+                                  (uint64_t((path >> 11) & 1u) << 44) | (uint64_t((path >> 12) & 1u) << 45) |
+                                  (uint64_t((path >> 13) & 1u) << 46) | (gbit << 47);
+            for (int k = 0; k < 6; ++k) codes[block * 6 + k] = uint8_t(word >> (8 * k));
+            if (cosine) cosine[block] = S.best_val / sqrtf(wn2);
+        }
+        __syncthreads();
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_encode(const float* w, const float* sigma, const void* table, unsigned char* codes, float* cosine,
+                          size_t nblocks, cudaStream_t s) {
+    static bool attr_set[64] = {false};
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const int smem = int(sizeof(EncShared));
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(k_encode, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    const unsigned grid = unsigned(nblocks < size_t(sms) ? nblocks : size_t(sms));
+    k_encode<<<grid, kEncThreads, smem, s>>>(w, sigma, static_cast<const DeviceTables*>(table), codes, cosine, nblocks);
+    return cudaGetLastError();
+}
+
+}  // namespace tetra

@@ -45,6 +45,10 @@ size_t batched_workspace_bytes(int N, int blocks_per_row);
 cudaError_t launch_gemv_batched(const void* codes, const float* row_scales, const void* table, const void* x,
                                 float* y, int N, int K, int batch, const void* tail, void* ws, cudaStream_t s);
 
+// Encoder search: per block of 24 weights the codebook point of largest cosine and the gain bit.
+cudaError_t launch_encode(const float* w, const float* sigma, const void* table, unsigned char* codes, float* cosine,
+                          size_t nblocks, cudaStream_t s);
+
 // Plan of a single product, for callers that bring their own scratch memory:
 // single_plan_fill writes single_plan_meta_bytes() bytes of plan data to a host
 // buffer; copied to the start of a scratch area of single_plan_scratch_bytes(blocks)

@@ -66,6 +66,7 @@ def lib():
         L.tetra_batched_workspace_bytes.restype = sz
         L.tetra_gemv_batched.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, sz, vp]
         L.tetra_gemv_noalloc.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, vp]
+        L.tetra_encode_blocks.argtypes = [vp, vp, vp, vp, vp, sz, vp]
         L.tetra_q4_packed_bytes.argtypes = [i32, i32, i32]
         L.tetra_q4_packed_bytes.restype = sz
         L.tetra_q4_pack.argtypes = [vp, vp, vp, vp, sz, i32, i32, i32, vp]
@@ -270,3 +271,13 @@ def tetra_q4_rows(packed, ids, out, N: int, K: int, G: int, stream=None):
     _check(lib().tetra_q4_rows(_ptr(packed), _ptr(ids), int(ids.numel()), _ptr(out), N, K, G, _stream(stream)),
            "tetra_q4_rows")
     return out
+
+
+def tetra_encode_blocks(w, table, sigma=None, want_cosine=True, stream=None):
+    """w: float32 [n, 24] on the device -> (codes uint8 [n, 6] in file order, cosines float32 [n] or None)."""
+    n = w.numel() // 24
+    codes = torch.empty((n, 6), dtype=torch.uint8, device=w.device)
+    cos = torch.empty(n, dtype=torch.float32, device=w.device) if want_cosine else None
+    _check(lib().tetra_encode_blocks(_ptr(w), _ptr(sigma), _ptr(table), _ptr(codes), _ptr(cos), n, _stream(stream)),
+           "tetra_encode_blocks")
+    return codes, cos

@@ -1,0 +1,90 @@
+"""GPU parity of the encoder search against the exact-search oracle, through the C ABI (Sec. 3.1, Eq. (2)).
+
+The objective has a unique VALUE (the largest cosine over the codebook); the word that attains it is unique
+only up to ties and float32 rounding of near-ties, so the test compares the value and checks that the word the
+GPU returns is valid: decoded by the oracle's decoder it attains, in FP64, the oracle's optimum within the
+float32 rounding of a 24-term correlation (1e-5 relative)."""
+import numpy as np
+import pytest
+
+from paper_2609_35465_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+MASK47 = np.uint64((1 << 47) - 1)
+
+
+def _encode_gpu(w, sigma=None):
+    import torch
+    from paper_2609_35465_b200 import tetra
+    table = tetra.tetra_build_table(synth.DEFAULT_GAIN)
+    wd = torch.from_numpy(np.ascontiguousarray(w, dtype=np.float32)).cuda()
+    sd = None if sigma is None else torch.from_numpy(np.ascontiguousarray(sigma, dtype=np.float32)).cuda()
+    codes, cos = tetra.tetra_encode_blocks(wd, table, sd)
+    torch.cuda.synchronize()
+    return synth.bytes_to_words(codes.cpu().numpy()), cos.cpu().numpy().astype(np.float64)
+
+
+def _fp64_cosine(orc, words, w):
+    Y, m, g = orc.decode_blocks(synth.words_to_bytes(words))
+    Y = Y.astype(np.float64)
+    return (Y * w).sum(1) / (np.linalg.norm(Y, axis=1) * np.linalg.norm(w, axis=1)), Y, g
+
+
+def test_encode_matches_exact_search(orc):
+    from oracle import encode as oe
+    n = 192
+    w = synth.normal(41, 0, 20, n * 24).reshape(n, 24).astype(np.float32)
+    w[5] *= 1e-3          # scale must not matter
+    w[6] *= 1e3
+    w[7, 8:] = 0          # mass in one section
+    w[8] = -np.abs(w[8])  # one orthant
+    words, cos = _encode_gpu(w)
+    w64 = w.astype(np.float64)
+    _, want = oe.encode_blocks(w64)
+    got, Y, _ = _fp64_cosine(orc, words, w64)
+    assert np.all(np.isfinite(got))
+    assert np.max(np.abs(got - want) / want) <= 1e-5     # the returned word attains the optimum
+    assert np.all(got <= want + 1e-12)                   # and nothing beats the exact search
+    assert np.max(np.abs(cos - got)) <= 1e-5             # the cosine it reports is the word's
+    for y in Y[:32]:
+        assert orc.in_leech(y.astype(np.int8))
+
+
+def test_encode_round_trip_and_zero_block(orc):
+    wds = synth.words(42, 0, 64)
+    Y, m, g = orc.decode_blocks(synth.words_to_bytes(wds))
+    Y = Y[m > 0].astype(np.float32)
+    Y = np.concatenate([Y, np.zeros((1, 24), np.float32)])
+    words, cos = _encode_gpu(Y)
+    assert words[-1] == 0 and cos[-1] == 0.0
+    assert np.all(cos[:-1] >= 1 - 1e-6)
+    got, _, _ = _fp64_cosine(orc, words[:-1], Y[:-1].astype(np.float64))
+    assert np.all(got >= 1 - 1e-12)   # a codebook point encodes to a point of the same direction
+
+
+def test_encode_gain_bit_follows_the_rule(orc):
+    from oracle import encode as oe
+    n = 256
+    w = synth.normal(43, 0, 20, n * 24).reshape(n, 24).astype(np.float32)
+    sigma = np.exp(synth.normal(43, 1, 20, n) * 0.2).astype(np.float32)
+    words, cos = _encode_gpu(w, sigma)
+    gain = synth.DEFAULT_GAIN.astype(np.float64)
+    got, Y, g = _fp64_cosine(orc, words, w.astype(np.float64))
+    c = got * np.linalg.norm(w.astype(np.float64), axis=1)
+    for i in range(n):
+        want = oe.choose_gain(c[i], float(sigma[i]), gain)
+        err = (gain * sigma[i]) ** 2 - 2 * gain * sigma[i] * c[i]
+        if abs(err[0] - err[1]) > 1e-4 * abs(err).max():   # away from the decision boundary
+            assert int(g[i]) == want
+    assert set(g.tolist()) == {0, 1}
+
+
+def test_encode_is_deterministic_and_handles_many_blocks(orc):
+    n = 1500   # more blocks than CTAs: the persistent loop
+    w = synth.normal(44, 0, 20, n * 24).reshape(n, 24).astype(np.float32)
+    a, ca = _encode_gpu(w)
+    b, cb = _encode_gpu(w)
+    assert np.array_equal(a, b) and np.array_equal(ca, cb)
+    got, _, _ = _fp64_cosine(orc, a, w.astype(np.float64))
+    assert got.min() > 0.9 and abs(got.mean() - 0.9608) < 0.003   # the exact search's mean cosine on Gaussian blocks
