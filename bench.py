@@ -176,6 +176,9 @@ def main():
     ap.add_argument("--batched-only", type=int, default=0, metavar="VECTORS",
                     help="profiling runs: two rounds of tetra_gemv_batched over 12 copies of the 4096 x 12288 "
                          "matrix with this many vectors, nothing else, no JSON line")
+    ap.add_argument("--encode-only", type=int, default=0, metavar="BLOCKS",
+                    help="profiling runs: two tetra_encode_blocks launches on this many Gaussian blocks, nothing else, "
+                         "no JSON line")
     ap.add_argument("--q4-only", default="", metavar="N,K,G,BATCH",
                     help="profiling runs: three tetra_q4_gemv launches on one synthetic matrix, nothing else, "
                          "no JSON line")
@@ -207,6 +210,15 @@ def main():
     elif not os.path.exists(tbuild.LIB) and not os.environ.get("TETRA_LIB"):
         tbuild.build()
 
+    if args.encode_only:
+        from paper_2609_35465_b200 import synth, tetra
+        ne = args.encode_only
+        wd = torch.from_numpy(synth.normal(11, 0, 20, ne * 24).reshape(ne, 24).astype(np.float32)).cuda()
+        enc_table = tetra.tetra_build_table(synth.DEFAULT_GAIN)
+        for _ in range(2):
+            tetra.tetra_encode_blocks(wd, enc_table)
+        torch.cuda.synchronize()
+        return
     if args.q4_only:
         from paper_2609_35465_b200 import synth, tetra
         qN, qK, qG, qB = (int(v) for v in args.q4_only.split(","))
@@ -420,6 +432,26 @@ def main():
             del packs, gg, qn, sc, of
             torch.cuda.empty_cache()
         out["q4_gemv"] = q4
+
+        # encoder search on Gaussian blocks (Sec. 3.5): exact largest-cosine point per block on the GPU, and the
+        # oracle's exact search on a bounded sample of the same blocks on the host cores
+        from oracle import encode as oenc
+        n_enc = 20000
+        w_enc = synth.normal(11, 0, 20, n_enc * 24).reshape(n_enc, 24).astype(np.float32)
+        wd = torch.from_numpy(w_enc).cuda()
+        enc_table = tetra.tetra_build_table(synth.DEFAULT_GAIN)
+        tetra.tetra_encode_blocks(wd, enc_table)
+        t_enc = timed(torch, lambda: tetra.tetra_encode_blocks(wd, enc_table), 3, 1, stream)
+        codes_enc, cos_enc = tetra.tetra_encode_blocks(wd, enc_table)
+        torch.cuda.synchronize()
+        t0 = time.time()
+        _, cos_ref = oenc.encode_blocks(w_enc[:256].astype(np.float64))
+        t_ref = time.time() - t0
+        out["encoder"] = {"blocks": n_enc, "ms": t_enc, "blocks_per_s": n_enc / (t_enc * 1e-3),
+                          "mean_cosine": float(cos_enc.mean().item()),
+                          "oracle_blocks_per_s": 256 / t_ref, "oracle_cores": os.cpu_count() or 1,
+                          "max_abs_cosine_difference_on_oracle_sample":
+                              float(np.max(np.abs(cos_enc[:256].cpu().numpy().astype(np.float64) - cos_ref)))}
 
         # the other two model sizes, planned-list pass (same kernels; a few repetitions)
         others = {}

@@ -88,3 +88,26 @@ def test_encode_is_deterministic_and_handles_many_blocks(orc):
     assert np.array_equal(a, b) and np.array_equal(ca, cb)
     got, _, _ = _fp64_cosine(orc, a, w.astype(np.float64))
     assert got.min() > 0.9 and abs(got.mean() - 0.9608) < 0.003   # the exact search's mean cosine on Gaussian blocks
+
+
+def test_encode_retention_at_full_size(orc):
+    """20,000 Gaussian blocks (Sec. 3.5): the GPU search reproduces what the exact-search oracle attains on the
+    same blocks (stored by tests/golden/make_encode_golden.py), which lies between the paper's two figures."""
+    import os
+    golden = {}
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "encode_retention.txt")):
+        if not line.startswith("#"):
+            k, v = line.split()
+            golden[k] = float(v)
+    n = int(golden["blocks"])
+    w = synth.normal(11, 0, 20, n * 24).reshape(n, 24).astype(np.float32)
+    words, cos = _encode_gpu(w)
+    got, Y, g = _fp64_cosine(orc, words, w.astype(np.float64))
+    gain = synth.DEFAULT_GAIN.astype(np.float64)
+    what = Y / np.linalg.norm(Y, axis=1, keepdims=True) * gain[g][:, None]
+    D = ((w.astype(np.float64) - what) ** 2).mean()
+    retention = 0.5 * np.log2(1.0 / D) / 2.0 * 100.0
+    assert abs(got.mean() - golden["mean_cosine"]) <= 1e-6
+    assert abs(got.min() - golden["min_cosine"]) <= 1e-5
+    assert abs(retention - golden["retention_percent"]) <= 2e-3
+    assert 88.80 <= retention <= 91.98
