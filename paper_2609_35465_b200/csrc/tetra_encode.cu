@@ -10,11 +10,12 @@
 //   * the sections are tied by the trellis path, by the parity and by Eq. (3) (r3 = p ^ r ^ delta): they are
 //     joined state by state with the summed norm and the class parity as extra state.
 // One CTA of 384 threads works on one block at a time: three groups of 128 threads, one per section, thread =
-// pattern byte.  For every batch of 64 rank rows a group first tabulates, per row, the partial correlations and
+// pattern byte.  For every batch of 32 rank rows a group tabulates, per row, the partial correlations and
 // norms of the 16 patterns of each half of the byte (so a (row, byte) candidate costs two shared loads and two
-// additions), then every thread scans the batch for its own byte and keeps the best correlation per (class,
-// k) in a private column of shared memory (no atomics).  The join runs on the same CTA; the rows that attain
-// the winning entries are found by a second scan of three lists.
+// additions) while every thread scans the batch before for its own byte and keeps the best correlation per
+// (class, k) in a private column of shared memory (no atomics; two columns, for even and odd rows, so that
+// two updates are in flight).  The join runs on the same CTA, every thread gathering a few entries of the
+// second cut; the rows that attain the winning entries are found by a second scan of three lists.
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -28,8 +29,8 @@ namespace tetra {
 namespace {
 
 constexpr int kEncThreads = 384;
-constexpr int kEncBatch = 64;       // rank rows per batch
-constexpr int kEncStride = 65;      // row-table entries are 65 rows apart (bank spread)
+constexpr int kEncBatch = 32;       // rank rows per batch
+constexpr int kEncStride = 33;      // row-table entries are 33 rows apart (bank spread)
 constexpr float kNeg = -1.0e30f;
 constexpr float kNegTest = -1.0e29f;
 
@@ -41,11 +42,10 @@ struct EncShared {
     uint16_t incoming[64][16];                 // per state after the branch: s8 | b2 << 6
     int incoming_count[64];
     float A[3][8][4][8];                       // w_j * value(o, rank)
-    uint2 rowtab[3][32 * kEncStride];          // (partial correlation, partial norm): entry (half * 16 + pattern), row
-    float T[3][20][128];                       // best correlation per (class * 10 + k), byte
+    uint2 rowtab[2][3][32 * kEncStride];       // two buffers of (partial correlation, partial norm): entry (half * 16 + pattern), row
+    float T[3][2][20][128];                    // best correlation per (class * 10 + k), byte; one copy for even, one for odd rows
     float F1[64][2][20];                       // after section 1: state, class, norm / 8
     float H[39][128];                          // after section 2: norm / 8, (state after the branch) * 2 + class parity
-    uint32_t Hback[39][128];
     float red_val[kEncThreads / 32];
     uint32_t red_arg[kEncThreads / 32];
     float w[24];
@@ -169,59 +169,76 @@ k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const Dev
 
         for (int p = 0; p < 2; ++p) {
             // ---------------- section tables ----------------
-            for (int i = ct; i < 20 * 128; i += 128) (&S.T[sg][0][0])[i] = kNeg;
-            group_barrier(sg);
-            for (int cls = 0; cls < 2; ++cls) {
-                const int len = list_length(sg, cls), base = 2048 * cls;
-                for (int b0 = 0; b0 < len; b0 += kEncBatch) {
-                    const int nb = min(kEncBatch, len - b0);
-                    if (ct < nb) {  // tabulate one row: 16 patterns of each half of the byte
-                        const uint32_t rw = S.rows[base + b0 + ct];
+            for (int i = ct; i < 2 * 20 * 128; i += 128) (&S.T[sg][0][0][0])[i] = kNeg;
+            // thread (row of the batch = ct / 2, half of the byte = ct & 1) tabulates 16 patterns while the whole
+            // group scans the batch before: one barrier per batch
+            auto produce = [&](int buf, int cls, int b0) {
+                const int len = list_length(sg, cls);
+                const int r = ct >> 1, half = ct & 1;
+                if (ct < 2 * kEncBatch && b0 + r < len) {
+                    const uint32_t rw = S.rows[2048 * cls + b0 + r];
+                    float P[16];
+                    int Nn[16];
+                    P[0] = 0.f;
+                    Nn[0] = 0;
+                    float d[4];
+                    int dn[4];
 #pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            float P[16];
-                            int Nn[16];
-                            P[0] = 0.f;
-                            Nn[0] = 0;
-                            float d[4];
-                            int dn[4];
+                    for (int jj = 0; jj < 4; ++jj) {
+                        const int j = 4 * half + jj, rho = (rw >> (4 * j)) & 7;
+                        const float a0 = S.A[sg][j][p][rho], a1 = S.A[sg][j][p + 2][rho];
+                        const int v0 = rank_value(p, rho), v1 = rank_value(p + 2, rho);
+                        P[0] += a0;
+                        Nn[0] += v0 * v0;
+                        d[jj] = a1 - a0;
+                        dn[jj] = v1 * v1 - v0 * v0;
+                    }
 #pragma unroll
-                            for (int jj = 0; jj < 4; ++jj) {
-                                const int j = 4 * half + jj, rho = (rw >> (4 * j)) & 7;
-                                const float a0 = S.A[sg][j][p][rho], a1 = S.A[sg][j][p + 2][rho];
-                                const int v0 = rank_value(p, rho), v1 = rank_value(p + 2, rho);
-                                P[0] += a0;
-                                Nn[0] += v0 * v0;
-                                d[jj] = a1 - a0;
-                                dn[jj] = v1 * v1 - v0 * v0;
-                            }
+                    for (int jj = 0; jj < 4; ++jj)
 #pragma unroll
-                            for (int jj = 0; jj < 4; ++jj)
-#pragma unroll
-                                for (int m = 0; m < (1 << jj); ++m) {
-                                    P[m | (1 << jj)] = P[m] + d[jj];
-                                    Nn[m | (1 << jj)] = Nn[m] + dn[jj];
-                                }
-#pragma unroll
-                            for (int m = 0; m < 16; ++m)
-                                S.rowtab[sg][(half * 16 + m) * kEncStride + ct] = make_uint2(__float_as_uint(P[m]), uint32_t(Nn[m]));
+                        for (int m = 0; m < (1 << jj); ++m) {
+                            P[m | (1 << jj)] = P[m] + d[jj];
+                            Nn[m | (1 << jj)] = Nn[m] + dn[jj];
                         }
-                    }
-                    group_barrier(sg);
-                    const uint2* lo_tab = &S.rowtab[sg][my_lo * kEncStride];
-                    const uint2* hi_tab = &S.rowtab[sg][(16 + my_hi) * kEncStride];
-                    float* my_t = &S.T[sg][cls * 10][ct];
-#pragma unroll 4
-                    for (int r = 0; r < nb; ++r) {
-                        const uint2 lo = lo_tab[r], hi = hi_tab[r];
-                        const float corr = __uint_as_float(lo.x) + __uint_as_float(hi.x);
-                        const int k = int(lo.y + hi.y) >> 4;
-                        float* cell = my_t + k * 128;
-                        *cell = fmaxf(*cell, corr);
-                    }
-                    group_barrier(sg);
+#pragma unroll
+                    for (int m = 0; m < 16; ++m)
+                        S.rowtab[buf][sg][(half * 16 + m) * kEncStride + r] = make_uint2(__float_as_uint(P[m]), uint32_t(Nn[m]));
                 }
+            };
+            // the batches of both classes as one sequence
+            const int nb0 = (list_length(sg, 0) + kEncBatch - 1) / kEncBatch, nb1 = (list_length(sg, 1) + kEncBatch - 1) / kEncBatch;
+            produce(0, 0, 0);
+            group_barrier(sg);
+            for (int bi = 0; bi < nb0 + nb1; ++bi) {
+                const int buf = bi & 1;
+                const int cls = bi < nb0 ? 0 : 1, b0 = (bi < nb0 ? bi : bi - nb0) * kEncBatch;
+                if (bi + 1 < nb0 + nb1) {
+                    const int nbi = bi + 1;
+                    produce(buf ^ 1, nbi < nb0 ? 0 : 1, (nbi < nb0 ? nbi : nbi - nb0) * kEncBatch);
+                }
+                const int nb = min(kEncBatch, list_length(sg, cls) - b0);
+                const uint2* lo_tab = &S.rowtab[buf][sg][my_lo * kEncStride];
+                const uint2* hi_tab = &S.rowtab[buf][sg][(16 + my_hi) * kEncStride];
+                float* t_even = &S.T[sg][0][cls * 10][ct];
+                float* t_odd = &S.T[sg][1][cls * 10][ct];
+                int r = 0;
+                for (; r + 1 < nb; r += 2) {  // two independent read-modify-write chains
+                    const uint2 lo0 = lo_tab[r], hi0 = hi_tab[r], lo1 = lo_tab[r + 1], hi1 = hi_tab[r + 1];
+                    float* c0 = t_even + (int(lo0.y + hi0.y) >> 4) * 128;
+                    float* c1 = t_odd + (int(lo1.y + hi1.y) >> 4) * 128;
+                    const float v0 = *c0, v1 = *c1;
+                    *c0 = fmaxf(v0, __uint_as_float(lo0.x) + __uint_as_float(hi0.x));
+                    *c1 = fmaxf(v1, __uint_as_float(lo1.x) + __uint_as_float(hi1.x));
+                }
+                if (r < nb) {
+                    const uint2 lo0 = lo_tab[r], hi0 = hi_tab[r];
+                    float* c0 = t_even + (int(lo0.y + hi0.y) >> 4) * 128;
+                    *c0 = fmaxf(*c0, __uint_as_float(lo0.x) + __uint_as_float(hi0.x));
+                }
+                group_barrier(sg);
             }
+            for (int i = ct; i < 20 * 128; i += 128)  // fold the odd rows' copy into the even rows'
+                (&S.T[sg][0][0][0])[i] = fmaxf((&S.T[sg][0][0][0])[i], (&S.T[sg][1][0][0])[i]);
             __syncthreads();
 
             // ---------------- join: first cut ----------------
@@ -232,35 +249,49 @@ k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const Dev
                 for (int b1 = 0; b1 < 2; ++b1) {
                     const int byte = S.prefixes[2 * s8 + b1];
                     const int rem = 8 * n8 - norm_residue(p, cls, byte);
-                    if (rem >= 0 && (rem & 15) == 0 && (rem >> 4) < 10) best = fmaxf(best, S.T[0][cls * 10 + (rem >> 4)][even_index(byte)]);
+                    if (rem >= 0 && (rem & 15) == 0 && (rem >> 4) < 10) best = fmaxf(best, S.T[0][0][cls * 10 + (rem >> 4)][even_index(byte)]);
                 }
                 S.F1[s8][cls][n8] = best;
             }
-            for (int e = tid; e < 39 * 128; e += kEncThreads) (&S.H[0][0])[e] = kNeg;
             __syncthreads();
             // ---------------- second cut ----------------
+            // thread = (state after the branch, class parity): all 39 entries of its column are accumulated in
+            // registers (two sets, for the two possible norm residues of section 2's byte) over the 16 branches
+            // into the state, the class of section 1, the 20 norms after section 1 and the 10 of section 2
             if (tid < 128) {
                 const int s16 = tid >> 1, par = tid & 1;
+                float h0[38], h1[38];  // index n8 + 2 k2, residue 0 / 8 of section 2
+#pragma unroll
+                for (int i = 0; i < 38; ++i) h0[i] = h1[i] = kNeg;
                 for (int in = 0; in < 16; ++in) {
-                    const int sb = S.incoming[s16][in], s8 = sb >> 4, b2 = sb & 15;
+                    const int sb = S.incoming[s16][in], s8 = sb >> 4;
                     const int byte2 = S.branches[sb] & 0xFF, ci2 = even_index(byte2);
                     for (int cls1 = 0; cls1 < 2; ++cls1) {
-                        const int cls2 = par ^ cls1, res2 = norm_residue(p, cls2, byte2) >> 3;
-                        for (int n8 = 0; n8 < 20; ++n8) {
-                            const float a = S.F1[s8][cls1][n8];
-                            if (a < kNegTest) continue;
+                        const int cls2 = par ^ cls1;
+                        float a[20], b[10];
 #pragma unroll
-                            for (int k2 = 0; k2 < 10; ++k2) {
-                                const float b = S.T[1][cls2 * 10 + k2][ci2];
-                                const int q = n8 + 2 * k2 + res2;
-                                if (b > kNegTest && a + b > S.H[q][tid]) {
-                                    S.H[q][tid] = a + b;
-                                    S.Hback[q][tid] = uint32_t(s8) | (uint32_t(b2) << 6) | (uint32_t(cls1) << 10) |
-                                                      (uint32_t(n8) << 11) | (uint32_t(k2) << 16);
-                                }
-                            }
+                        for (int n8 = 0; n8 < 20; ++n8) a[n8] = S.F1[s8][cls1][n8];
+#pragma unroll
+                        for (int k2 = 0; k2 < 10; ++k2) b[k2] = S.T[1][0][cls2 * 10 + k2][ci2];
+                        if (norm_residue(p, cls2, byte2)) {
+#pragma unroll
+                            for (int n8 = 0; n8 < 20; ++n8)
+#pragma unroll
+                                for (int k2 = 0; k2 < 10; ++k2) h1[n8 + 2 * k2] = fmaxf(h1[n8 + 2 * k2], a[n8] + b[k2]);
+                        } else {
+#pragma unroll
+                            for (int n8 = 0; n8 < 20; ++n8)
+#pragma unroll
+                                for (int k2 = 0; k2 < 10; ++k2) h0[n8 + 2 * k2] = fmaxf(h0[n8 + 2 * k2], a[n8] + b[k2]);
                         }
                     }
+                }
+                // an absent entry stays far below every real one (sums of two absent entries are more negative still)
+#pragma unroll
+                for (int q = 0; q < 39; ++q) {
+                    float v = q < 38 ? h0[q] : kNeg;
+                    if (q >= 1) v = fmaxf(v, h1[q - 1]);
+                    S.H[q][tid] = v > kNegTest ? v : kNeg;
                 }
             }
             __syncthreads();
@@ -276,7 +307,7 @@ k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const Dev
                     if (a < kNegTest) continue;
 #pragma unroll
                     for (int k3 = 0; k3 < 10; ++k3) {
-                        const float b = S.T[2][cls3 * 10 + k3][ci3];
+                        const float b = S.T[2][0][cls3 * 10 + k3][ci3];
                         const int n = 8 * q + 16 * k3 + res3;
                         if (b > kNegTest && n > 0) {
                             const float v = (a + b) / sqrtf(float(n));
@@ -293,7 +324,29 @@ k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const Dev
             if (val > S.best_val) {  // uniform: resolve the path and the rows while this parity's tables are alive
                 const int wt = int(arg >> 16), q = int(arg >> 8) & 0xFF, k3 = int(arg & 0xFF);
                 const int s16 = wt >> 2, b3 = (wt >> 1) & 1, par = wt & 1;
-                const uint32_t back = S.Hback[q][s16 * 2 + par];
+                // which branch, class and norms attain the winning entry of the second cut: the first, in (branch,
+                // class, norm) order, whose sum is the entry (the same additions as above, so the match is exact)
+                uint32_t back = 0;
+                {
+                    const float target = S.H[q][s16 * 2 + par];
+                    bool found = false;
+                    for (int in = 0; in < 16 && !found; ++in) {
+                        const int sb = S.incoming[s16][in], s8c = sb >> 4, b2c = sb & 15;
+                        const int byte2 = S.branches[sb] & 0xFF, ci2 = even_index(byte2);
+                        for (int c1 = 0; c1 < 2 && !found; ++c1) {
+                            const int c2 = par ^ c1, res2 = norm_residue(p, c2, byte2) >> 3;
+                            for (int kk = 0; kk < 10 && !found; ++kk) {
+                                const int n8c = q - 2 * kk - res2;
+                                if (n8c < 0 || n8c >= 20) continue;
+                                if (S.F1[s8c][c1][n8c] + S.T[1][0][c2 * 10 + kk][ci2] == target) {
+                                    back = uint32_t(s8c) | (uint32_t(b2c) << 6) | (uint32_t(c1) << 10) |
+                                           (uint32_t(n8c) << 11) | (uint32_t(kk) << 16);
+                                    found = true;
+                                }
+                            }
+                        }
+                    }
+                }
                 const int s8 = back & 63, b2 = (back >> 6) & 15, cls1 = (back >> 10) & 1, n8 = (back >> 11) & 31,
                           k2 = (back >> 16) & 15;
                 const int cls2 = par ^ cls1, cls3 = p ^ par;
@@ -305,7 +358,7 @@ k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const Dev
                         const int byte = S.prefixes[2 * s8 + bb];
                         const int rem = 8 * n8 - norm_residue(p, cls1, byte);
                         if (rem >= 0 && (rem & 15) == 0 && (rem >> 4) < 10) {
-                            const float v = S.T[0][cls1 * 10 + (rem >> 4)][even_index(byte)];
+                            const float v = S.T[0][0][cls1 * 10 + (rem >> 4)][even_index(byte)];
                             if (v > bestv) {
                                 bestv = v;
                                 b1 = bb;
