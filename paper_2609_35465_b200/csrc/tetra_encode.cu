@@ -42,6 +42,7 @@ struct EncShared {
     uint16_t incoming[64][16];                 // per state after the branch: s8 | b2 << 6
     int incoming_count[64];
     float A[3][8][4][8];                       // w_j * value(o, rank)
+    int V2[4][8];                              // value(o, rank)^2
     uint2 rowtab[2][3][32 * kEncStride];       // two buffers of (partial correlation, partial norm): entry (half * 16 + pattern), row
     float T[3][2][20][128];                    // best correlation per (class * 10 + k), byte; one copy for even, one for odd rows
     float F1[64][2][20];                       // after section 1: state, class, norm / 8
@@ -120,6 +121,7 @@ k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const Dev
         S.suffixes[tid] = tab->paper.suffixes[tid];
     }
     if (tid < 64) S.incoming_count[tid] = 0;
+    if (tid < 32) S.V2[tid >> 3][tid & 7] = rank_value(tid >> 3, tid & 7) * rank_value(tid >> 3, tid & 7);
     __syncthreads();
     for (int i = tid; i < 1024; i += kEncThreads) {  // order within a state's list does not matter for the maximum,
         const int s16 = S.branches[i] >> 8;          // but it decides ties: sort below
@@ -187,11 +189,11 @@ k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const Dev
                     for (int jj = 0; jj < 4; ++jj) {
                         const int j = 4 * half + jj, rho = (rw >> (4 * j)) & 7;
                         const float a0 = S.A[sg][j][p][rho], a1 = S.A[sg][j][p + 2][rho];
-                        const int v0 = rank_value(p, rho), v1 = rank_value(p + 2, rho);
+                        const int n0 = S.V2[p][rho], n1 = S.V2[p + 2][rho];
                         P[0] += a0;
-                        Nn[0] += v0 * v0;
+                        Nn[0] += n0;
                         d[jj] = a1 - a0;
-                        dn[jj] = v1 * v1 - v0 * v0;
+                        dn[jj] = n1 - n0;
                     }
 #pragma unroll
                     for (int jj = 0; jj < 4; ++jj)
@@ -202,7 +204,7 @@ k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const Dev
                         }
 #pragma unroll
                     for (int m = 0; m < 16; ++m)
-                        S.rowtab[buf][sg][(half * 16 + m) * kEncStride + r] = make_uint2(__float_as_uint(P[m]), uint32_t(Nn[m]));
+                        S.rowtab[buf][sg][(half * 16 + m) * kEncStride + r] = make_uint2(__float_as_uint(P[m]), uint32_t(Nn[m]) * 32u);
                 }
             };
             // the batches of both classes as one sequence
@@ -219,21 +221,33 @@ k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const Dev
                 const int nb = min(kEncBatch, list_length(sg, cls) - b0);
                 const uint2* lo_tab = &S.rowtab[buf][sg][my_lo * kEncStride];
                 const uint2* hi_tab = &S.rowtab[buf][sg][(16 + my_hi) * kEncStride];
-                float* t_even = &S.T[sg][0][cls * 10][ct];
-                float* t_odd = &S.T[sg][1][cls * 10][ct];
-                int r = 0;
-                for (; r + 1 < nb; r += 2) {  // two independent read-modify-write chains
-                    const uint2 lo0 = lo_tab[r], hi0 = hi_tab[r], lo1 = lo_tab[r + 1], hi1 = hi_tab[r + 1];
-                    float* c0 = t_even + (int(lo0.y + hi0.y) >> 4) * 128;
-                    float* c1 = t_odd + (int(lo1.y + hi1.y) >> 4) * 128;
-                    const float v0 = *c0, v1 = *c1;
-                    *c0 = fmaxf(v0, __uint_as_float(lo0.x) + __uint_as_float(hi0.x));
-                    *c1 = fmaxf(v1, __uint_as_float(lo1.x) + __uint_as_float(hi1.x));
-                }
-                if (r < nb) {
-                    const uint2 lo0 = lo_tab[r], hi0 = hi_tab[r];
-                    float* c0 = t_even + (int(lo0.y + hi0.y) >> 4) * 128;
-                    *c0 = fmaxf(*c0, __uint_as_float(lo0.x) + __uint_as_float(hi0.x));
+                // a candidate's cell: the tables hold 32 x norm, a column's cells are 512 bytes apart and the norm is
+                // 16 k + residue, so  cell = column + 32 norm - 32 residue  (one three-input addition)
+                const uint32_t res32 = uint32_t(norm_residue(p, cls, my_byte)) * 32u;
+                const uint32_t t_even = smem_u32(&S.T[sg][0][cls * 10][ct]) - res32;
+                const uint32_t t_odd = smem_u32(&S.T[sg][1][cls * 10][ct]) - res32;
+                auto update = [&](uint32_t column, uint2 lo, uint2 hi) {
+                    const uint32_t cell = column + lo.y + hi.y;
+                    float v;
+                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(cell));
+                    v = fmaxf(v, __uint_as_float(lo.x) + __uint_as_float(hi.x));
+                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(cell), "f"(v) : "memory");
+                };
+                if (nb == kEncBatch) {
+#pragma unroll
+                    for (int r = 0; r < kEncBatch; r += 2) {  // two independent read-modify-write chains, loads first
+                        const uint2 lo0 = lo_tab[r], hi0 = hi_tab[r], lo1 = lo_tab[r + 1], hi1 = hi_tab[r + 1];
+                        const uint32_t cell0 = t_even + lo0.y + hi0.y, cell1 = t_odd + lo1.y + hi1.y;
+                        float v0, v1;
+                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v0) : "r"(cell0));
+                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v1) : "r"(cell1));
+                        v0 = fmaxf(v0, __uint_as_float(lo0.x) + __uint_as_float(hi0.x));
+                        v1 = fmaxf(v1, __uint_as_float(lo1.x) + __uint_as_float(hi1.x));
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(cell0), "f"(v0) : "memory");
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(cell1), "f"(v1) : "memory");
+                    }
+                } else {
+                    for (int r = 0; r < nb; ++r) update(t_even, lo_tab[r], hi_tab[r]);
                 }
                 group_barrier(sg);
             }
