@@ -107,7 +107,6 @@ constexpr int kRedStride = 36;                 // floats per row of the transpos
 constexpr int kRedFloats = 8 * kRedStride;     // per warp
 constexpr int kRowAccFloats = 2048;            // k_gemv_fast: per-CTA buffer of per-(column group, row) sums
 constexpr int kXqBytesPerCol = 80;             // 3 planes x 24 bytes, step, sum
-constexpr uint32_t kXqHi = 0, kXqMid = 24, kXqLo = 48;
 
 struct LaneX {
     uint32_t hi[6];   // bits 23..16 of q (signed), int8 x 4
