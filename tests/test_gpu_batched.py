@@ -36,7 +36,7 @@ def run(tt, table, m):
 @pytest.mark.parametrize("N,K,tail_mode,batch", [
     (256, 2560, True, 2), (256, 2560, True, 5), (256, 2560, True, 8), (256, 2560, True, 16),
     (520, 4096, True, 16), (33, 24 * 31 + 5, True, 3), (33, 24 * 31 + 5, False, 9), (7, 48, True, 16),
-    (1, 24, True, 1), (72, 17408, True, 12), (2048, 2304, True, 4),
+    (1, 24, True, 1), (72, 17408, True, 12), (2048, 2304, True, 4), (40, 49152, True, 3), (24, 49152, True, 16),
 ])
 def test_batched_matches_oracle(tt, table, orc, N, K, tail_mode, batch):
     m = make_matrix(51, N * 3 + K + batch, N, K, tail_mode, batch=batch)

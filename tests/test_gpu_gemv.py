@@ -58,6 +58,8 @@ CASES = [
     (33, 24 * 31 + 5, True),
     (33, 24 * 31 + 5, False),
     (300, 24 * 513, True),
+    (40, 49152, True),          # the largest K the library takes (2048 blocks per row)
+    (17, 49152 - 7, False),
 ]
 
 
@@ -119,6 +121,7 @@ def test_grouped_launch_one_layer(tt, table, orc):
     [(512, 2560, True), (264, 12288, True), (72, 17408, True), (9, 24 * 33, True)],   # a few matrices
     [(1024, 4096, True)],                                                             # a single one
     [(33, 24 * 31 + 5, False), (7, 48, True), (1, 24, True)],                         # tiny and ragged
+    [(40, 49152, True), (3000, 24 * 64, True), (16, 49152 - 24, True)],               # the largest K, coarse mode
 ])
 def test_grouped_small_lists(tt, table, orc, shapes_list):
     """Small lists run in the planned path's fine mode (one row group x a slice of the column
