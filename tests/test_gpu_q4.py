@@ -44,6 +44,7 @@ def _check_gemv(q, scale, offset, packed, x, N, K, G, batch):
     (16, 128, 128, 1), (16, 64, 64, 1), (64, 1024, 128, 1), (37, 1152, 128, 1), (1, 256, 64, 1),
     (1024, 4096, 128, 1), (2560, 9728, 128, 1), (300, 4096, 64, 1), (512, 17408, 128, 1),
     (129, 2560, 64, 3), (256, 4096, 128, 8), (2048, 5120, 64, 5),
+    (64, 32768, 64, 1), (48, 65536, 128, 2), (40, 65536, 64, 1),   # the largest K the library takes
 ])
 def test_q4_gemv_matches_oracle(N, K, G, batch):
     q, s, o, packed = _device_matrix(21, N + K, N, K, G)
