@@ -335,8 +335,21 @@ def main():
         assert np.linalg.norm(y_single - y_grouped) <= 1e-5 * np.linalg.norm(y_grouped), \
             "per-matrix launches differ from the planned run"
         arms["paper_design_stream_ms"] = timed(torch, dp.run_paper_design, max(3, reps // 5), 2, stream)
+        # 20 rounds of ten planned passes each: median and best round (the paper reports the median of its rounds)
+        rounds = sorted(timed(torch, dp.run_grouped, 10, 0, stream) for _ in range(20))
+        out["rounds_of_10_steps"] = {"median_ms": rounds[len(rounds) // 2], "best_ms": rounds[0], "worst_ms": rounds[-1]}
+        # launch-overhead control (Sec. 5.2's "no weights" arm): the same 252 single-matrix launches on
+        # matrices cut down to one block and a 16-weight tail per row (K = 40), i.e. next to no code reads
+        ctl = DevicePass([shapes.Matrix(m.name, m.N, 40) for m in mats], seed=args.seed + 19)
+        arms["no_weights_control_stream_ms"] = timed(torch, ctl.run_per_matrix, reps, 3, stream)
+        gc = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gc, stream=torch.cuda.Stream()):
+            ctl.run_per_matrix(stream=torch.cuda.current_stream())
+        arms["no_weights_control_graph_ms"] = timed(torch, gc.replay, reps, 3, stream)
+        del gc, ctl
         for k in list(arms):
-            arms[k.replace("_ms", "_GBps")] = dp.algorithmic_bytes / (arms[k] * 1e-3) / 1e9
+            if not k.startswith("no_weights"):
+                arms[k.replace("_ms", "_GBps")] = dp.algorithmic_bytes / (arms[k] * 1e-3) / 1e9
         out["other_arms"] = arms
         dp.run_grouped()
         torch.cuda.synchronize()
@@ -392,6 +405,11 @@ def main():
             sweep[str(batch)] = {"batched_us": us["batched"], "per_vector_launches_us": us["per_vector"],
                                  "us_per_vector": us["batched"] / batch,
                                  "weights_x_vectors_per_s": m.N * m.K * batch / us["batched"] * 1e6}
+        t1 = sweep["1"]
+        sweep["first_batch_over_1p25x_batch1_time"] = {
+            "batched": next((b for b in shapes.CONFIG4_BATCHES if sweep[str(b)]["batched_us"] > 1.25 * t1["batched_us"]), None),
+            "per_vector_launches": next((b for b in shapes.CONFIG4_BATCHES
+                                         if sweep[str(b)]["per_vector_launches_us"] > 1.25 * t1["per_vector_launches_us"]), None)}
         out["batch_sweep_4096x12288"] = sweep
         del one, ws
 
@@ -482,6 +500,9 @@ def main():
                                "gpu_vs_oracle_worst_fraction_of_tolerance": worst}
         if worst is not None and worst > 1.0:
             raise SystemExit("GPU result outside the tolerance on the CPU-baseline sample: %.3f" % worst)
+        dts, nbs, _, nms = oracle_sample(dp, orc, 1, 1)
+        out["cpu_baseline_single_thread"] = {"value": nbs / dts / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                             "sample": "first layer (%d matrices, %.3f GB), %.1f s" % (nms, nbs / 1e9, dts)}
 
     print(json.dumps(out))
     if world > 1:
