@@ -39,8 +39,8 @@ cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, 
 cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s);
 
 
-// 2..16 activation vectors at once (decode once, tensor-core contraction per block); ws holds the
-// vectors' fixed-point image, arrival counters and partial results: batched_workspace_bytes(N, words per row).
+// 1..16 activation vectors at once (decode once, tensor-core contraction per block); ws holds the partial
+// results of the CTAs' column ranges: batched_workspace_bytes(N, words per row).
 size_t batched_workspace_bytes(int N, int blocks_per_row);
 cudaError_t launch_gemv_batched(const void* codes, const float* row_scales, const void* table, const void* x,
                                 float* y, int N, int K, int batch, const void* tail, void* ws, cudaStream_t s);
