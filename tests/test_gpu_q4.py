@@ -123,3 +123,29 @@ def test_q4_argument_checks():
     out = torch.full((3, K), 1.0, dtype=torch.float16, device="cuda")
     tetra.tetra_q4_rows(packed, ids, out, N, K, G)
     assert torch.count_nonzero(out[1:]) == 0 and torch.count_nonzero(out[0]) > 0
+
+
+def test_q4_head_full_size_sampled_rows():
+    """The output-head shape the bench times (151,936 x 4096, groups of 64), batch 1 and 8: rows sampled over
+    the whole table (first, last, strip and CTA-range boundaries included) against the oracle."""
+    import torch
+    from oracle import q4 as oq
+    from paper_2609_35465_b200 import tetra
+    N, K, G = 151936, 4096, 64
+    q = synth.q4_nibbles(26, 1, N, K)
+    s, o = synth.q4_scales_offsets(26, 1, N, K // G)
+    packed = tetra.tetra_q4_pack(torch.from_numpy(q).cuda(), torch.from_numpy(s).cuda(), torch.from_numpy(o).cuda(),
+                                 N, K, G)
+    rng = np.random.default_rng(26)
+    rows = np.unique(np.concatenate([[0, 1, 31, 32, 33, 1023, 1024, 1056, N - 33, N - 32, N - 1],
+                                     rng.integers(0, N, 300)]))
+    for batch in (1, 8):
+        x = synth.activations(26, 2, K, batch)
+        y = torch.full((batch, N), float("nan"), dtype=torch.float32, device="cuda")
+        tetra.tetra_q4_gemv(packed, torch.from_numpy(x).cuda(), y, N, K, G, batch)
+        got = y.cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all()
+        want, tn = oq.gemv(q[rows], s[rows], o[rows], x, len(rows), K, G, batch)
+        d = got[:, rows] - want
+        assert np.linalg.norm(d) / np.linalg.norm(want) <= REL_L2
+        assert np.max(np.abs(d) / (ABS_COEF * tn + ABS_FLOOR)) <= 1.0
