@@ -196,7 +196,13 @@ int tetra_gemv_hostio(const void *codes, const float *row_scales, const void *ta
 /* A planned run with host activations and results: copies x_bytes from x_host to
  * x_dev, runs tetra_gemv_grouped_run, copies y_bytes from y_dev to y_host, all on
  * `stream`.  The planned problems' x and y pointers are expected to point into
- * [x_dev, x_dev + x_bytes) and [y_dev, y_dev + y_bytes).  Does not synchronise. */
+ * [x_dev, x_dev + x_bytes) and [y_dev, y_dev + y_bytes).  Does not synchronise.
+ * Mapped results: a problem's y may also point into page-locked host memory that
+ * the device can address (cudaHostAlloc / cudaHostRegister under unified
+ * addressing); the kernels then store the results there directly, while they
+ * run.  For a list planned that way pass y_host = y_dev = NULL: only the
+ * activations are copied, and the results are in host memory once the stream
+ * has passed the run. */
 int tetra_gemv_grouped_hostio(void *workspace_dev, const void *table, const void *x_host,
                               void *x_dev, size_t x_bytes, float *y_host, const float *y_dev,
                               size_t y_bytes, void *stream);

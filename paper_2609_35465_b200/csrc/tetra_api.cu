@@ -247,13 +247,15 @@ int tetra_gemv_hostio(const void* codes, const float* row_scales, const void* ta
 
 int tetra_gemv_grouped_hostio(void* workspace_dev, const void* table, const void* x_host, void* x_dev,
                               size_t x_bytes, float* y_host, const float* y_dev, size_t y_bytes, void* stream) {
-    if (!workspace_dev || !table || !x_host || !x_dev || !y_host || !y_dev) return TETRA_ERR_NULL;
-    if (x_bytes == 0 || y_bytes == 0) return TETRA_ERR_SIZE;
+    if (!workspace_dev || !table || !x_host || !x_dev) return TETRA_ERR_NULL;
+    const bool mapped_results = !y_host && !y_dev;  // the plan's y pointers aim at page-locked host memory
+    if (!mapped_results && (!y_host || !y_dev)) return TETRA_ERR_NULL;
+    if (x_bytes == 0 || (!mapped_results && y_bytes == 0)) return TETRA_ERR_SIZE;
     if (!aligned(workspace_dev, 16) || !aligned(table, 16)) return TETRA_ERR_ALIGN;
     cudaStream_t s = as_stream(stream);
     if (cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return TETRA_ERR_CUDA;
     const int rc = tetra_gemv_grouped_run(workspace_dev, table, stream);
-    if (rc) return rc;
+    if (rc || mapped_results) return rc;
     return cuda_status(cudaMemcpyAsync(y_host, y_dev, y_bytes, cudaMemcpyDeviceToHost, s));
 }
 

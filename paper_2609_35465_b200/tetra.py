@@ -209,11 +209,13 @@ def tetra_gemv_hostio(codes, row_scales, table, x_host, y_host, x_stage, y_stage
            "tetra_gemv_hostio")
 
 
-def tetra_gemv_grouped_hostio(workspace, table, x_host, x_dev, y_host, y_dev, stream=None):
-    """A planned run with pinned host activations / results (one copy in, the kernels, one copy out)."""
+def tetra_gemv_grouped_hostio(workspace, table, x_host, x_dev, y_host=None, y_dev=None, stream=None):
+    """A planned run with pinned host activations / results (one copy in, the kernels, one copy out); with
+    y_host = y_dev = None the plan's y pointers are taken to aim at mapped pinned host memory (no copy out)."""
+    y_bytes = 0 if y_dev is None else y_dev.numel() * y_dev.element_size()
     _check(lib().tetra_gemv_grouped_hostio(_ptr(workspace), _ptr(table), _ptr(x_host), _ptr(x_dev),
                                            x_dev.numel() * x_dev.element_size(), _ptr(y_host), _ptr(y_dev),
-                                           y_dev.numel() * y_dev.element_size(), _stream(stream)),
+                                           y_bytes, _stream(stream)),
            "tetra_gemv_grouped_hostio")
 
 

@@ -92,6 +92,23 @@ class DevicePass:
         tetra.tetra_gemv_grouped_hostio(self.workspace, self.table, self.x_host, self.x_all,
                                         self.y_host, self.y_all, stream=stream)
 
+    def plan_mapped_results(self):
+        """A second plan of the same list whose results go straight to pinned host memory (y_mapped)."""
+        self.y_mapped = torch.zeros_like(self.y_host).pin_memory()
+        items = []
+        for it in self.items:
+            j = dict(it)
+            j["y"] = self.y_mapped[it["yoff"]:it["yoff"] + it["N"]]
+            items.append(j)
+        self.problems_mapped = tetra.make_problems(items)
+        self.workspace_mapped = torch.empty(max(16, tetra.tetra_grouped_workspace_bytes(self.problems_mapped)),
+                                            dtype=torch.uint8, device=self.device)
+        tetra.tetra_gemv_grouped_plan(self.problems_mapped, self.workspace_mapped)
+        torch.cuda.synchronize()
+
+    def run_grouped_mapped(self, stream=None):
+        tetra.tetra_gemv_grouped_hostio(self.workspace_mapped, self.table, self.x_host, self.x_all, stream=stream)
+
     # ---- host copies for the checker ---------------------------------------
     def host_inputs(self, index: int, rows: Optional[np.ndarray] = None):
         """File-order codes (regenerated from the seed), scales, x and tail of matrix

@@ -202,3 +202,21 @@ def test_hostio_entry_point(tt, table, orc):
     tt.tetra_gemv_hostio(d["codes"], d["row_scales"], table, xh, yh, xs, d["y"], m["N"], m["K"], 1, d["tail"])
     torch.cuda.synchronize()
     assert_gemv_close(yh.numpy()[0], oracle_product(orc, m, GAIN), "hostio")
+
+
+def test_hostio_mapped_results(tt, table, orc):
+    """Results stored straight into pinned host memory (the plan's y pointers aim there): same bits as the
+    staged copy, and within tolerance of the oracle."""
+    from paper_2609_35465_b200 import shapes
+    from paper_2609_35465_b200.workload import DevicePass
+    dp = DevicePass([shapes.Matrix("a", 520, 4096), shapes.Matrix("b", 264, 2560), shapes.Matrix("c", 33, 749)], seed=61)
+    dp.run_grouped_hostio()
+    torch.cuda.synchronize()
+    staged = dp.y_host.numpy().copy()
+    dp.plan_mapped_results()
+    dp.run_grouped_mapped()
+    torch.cuda.synchronize()
+    assert np.array_equal(dp.y_mapped.numpy(), staged)
+    for i, it in enumerate(dp.items):
+        ref = oracle_product(orc, dp.host_inputs(i), dp.gain)
+        assert_gemv_close(dp.y_mapped.numpy()[it["yoff"]:it["yoff"] + it["N"]], ref, it["name"])
