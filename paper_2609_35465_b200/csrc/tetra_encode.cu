@@ -233,7 +233,23 @@ k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const Dev
                     v = fmaxf(v, __uint_as_float(lo.x) + __uint_as_float(hi.x));
                     asm volatile("st.shared.f32 [%0], %1;" ::"r"(cell), "f"(v) : "memory");
                 };
-                if (nb == kEncBatch) {
+                // At odd parity every coordinate is +-(2 rank + 1) whatever the pattern byte, so a row's norm is its
+                // cost and the rows of a class come sorted by cost: nearly every batch has ONE norm, the same for
+                // all bytes, and its best correlation is a running maximum in a register.
+                const uint32_t n_first = lo_tab[0].y + hi_tab[0].y, n_last = lo_tab[nb - 1].y + hi_tab[nb - 1].y;
+                if (p == 1 && nb == kEncBatch && n_first == n_last) {
+                    float m0 = kNeg, m1 = kNeg;
+#pragma unroll
+                    for (int r = 0; r < kEncBatch; r += 2) {
+                        m0 = fmaxf(m0, __uint_as_float(lo_tab[r].x) + __uint_as_float(hi_tab[r].x));
+                        m1 = fmaxf(m1, __uint_as_float(lo_tab[r + 1].x) + __uint_as_float(hi_tab[r + 1].x));
+                    }
+                    const uint32_t cell = t_even + n_first;
+                    float v;
+                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(cell));
+                    v = fmaxf(v, fmaxf(m0, m1));
+                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(cell), "f"(v) : "memory");
+                } else if (nb == kEncBatch) {
 #pragma unroll
                     for (int r = 0; r < kEncBatch; r += 2) {  // two independent read-modify-write chains, loads first
                         const uint2 lo0 = lo_tab[r], hi0 = hi_tab[r], lo1 = lo_tab[r + 1], hi1 = hi_tab[r + 1];
