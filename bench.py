@@ -198,6 +198,7 @@ def main():
     from paper_2609_35465_b200 import ranks, shapes
     from paper_2609_35465_b200 import build as tbuild
     from paper_2609_35465_b200.workload import DevicePass
+    from paper_2609_35465_b200 import tetra as tetra_mod
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
@@ -343,6 +344,33 @@ def main():
         assert np.linalg.norm(y_single - y_grouped) <= 1e-5 * np.linalg.norm(y_grouped), \
             "per-matrix launches differ from the planned run"
         arms["paper_design_stream_ms"] = timed(torch, dp.run_paper_design, max(3, reps // 5), 2, stream)
+        # the pass as a model would issue it: per layer four planned lists in stream order (q, k, v | o | gate, up |
+        # down: the matrices inside a list share their input and are independent, the lists depend on each
+        # other), every list planned once, the whole sequence replayed from one CUDA graph
+        if not args.layers or args.layers >= 1:
+            seq = []
+            for lo in range(0, len(dp.items), 7):
+                for a, b in ((0, 3), (3, 4), (4, 6), (6, 7)):
+                    pr = tetra_mod.make_problems(dp.items[lo + a:lo + b])
+                    wsq = torch.empty(max(16, tetra_mod.tetra_grouped_workspace_bytes(pr)), dtype=torch.uint8, device="cuda")
+                    tetra_mod.tetra_gemv_grouped_plan(pr, wsq)
+                    seq.append((pr, wsq))
+            torch.cuda.synchronize()
+
+            def run_sequence(stream=None):
+                for _, wsq in seq:
+                    tetra_mod.tetra_gemv_grouped_run(wsq, dp.table, stream=stream)
+            run_sequence()
+            gs_ = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gs_, stream=torch.cuda.Stream()):
+                run_sequence(stream=torch.cuda.current_stream())
+            arms["layer_sequence_graph_ms"] = timed(torch, gs_.replay, reps, 3, stream)
+            arms["layer_sequence_stream_ms"] = timed(torch, run_sequence, reps, 3, stream)
+            out["layer_sequence"] = {"lists_per_pass": len(seq), "launches_per_pass": 2 * len(seq),
+                                     "note": "four dependent planned lists per layer (q,k,v | o | gate,up | down)"}
+            del gs_
+            dp.run_grouped()
+            torch.cuda.synchronize()
         # 20 rounds of ten planned passes each: median and best round (the paper reports the median of its rounds)
         rounds = sorted(timed(torch, dp.run_grouped, 10, 0, stream) for _ in range(20))
         out["rounds_of_10_steps"] = {"median_ms": rounds[len(rounds) // 2], "best_ms": rounds[0], "worst_ms": rounds[-1]}
