@@ -130,7 +130,8 @@ __device__ __forceinline__ void lane_x_from_words(const uint32_t q[20], bool act
 // One block: device word -> contribution scale_b * sum_j y_j x_j (Eq. (2) without
 // the row scale).
 template <bool HI>
-__device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint32_t w1pair, const LaneX& X) {
+__device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint32_t w1pair, const LaneX& X,
+                                             float addend = 0.f) {
     FastBlock fb;
     fast_decode<HI>(sm_tab, w0, w1pair, fb);
     int dh = 0, dm = 0, dl = 0, n2 = 0;
@@ -146,7 +147,7 @@ __device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint3
     // n2 = 16 m; the scale table holds gain[g] / sqrt(16 m) at 128 g + 4 m.  The index is masked into
     // the table, so the load stays aligned and in bounds whatever the inputs are.
     const float scale = lds32f(fb.goff | ((uint32_t(n2) >> 2) & 0x7Cu));
-    return float(dot) * (scale * X.step);
+    return fmaf(float(dot), scale * X.step, addend);  // addend: the caller's running sum (one FFMA)
 }
 
 // The eight blocks of one 48-byte record (rows 8G..8G+7 of one column).
@@ -160,6 +161,19 @@ __device__ __forceinline__ void record_values(uint32_t sm_tab, const uint4& a, c
     v[5] = block_value<true>(sm_tab, b.y, h.z, X);
     v[6] = block_value<false>(sm_tab, b.z, h.w, X);
     v[7] = block_value<true>(sm_tab, b.w, h.w, X);
+}
+
+// The same, added to the caller's eight running sums.
+__device__ __forceinline__ void record_accumulate(uint32_t sm_tab, const uint4& a, const uint4& b, const uint4& h,
+                                                  const LaneX& X, float acc[8]) {
+    acc[0] = block_value<false>(sm_tab, a.x, h.x, X, acc[0]);
+    acc[1] = block_value<true>(sm_tab, a.y, h.x, X, acc[1]);
+    acc[2] = block_value<false>(sm_tab, a.z, h.y, X, acc[2]);
+    acc[3] = block_value<true>(sm_tab, a.w, h.y, X, acc[3]);
+    acc[4] = block_value<false>(sm_tab, b.x, h.z, X, acc[4]);
+    acc[5] = block_value<true>(sm_tab, b.y, h.z, X, acc[5]);
+    acc[6] = block_value<false>(sm_tab, b.z, h.w, X, acc[6]);
+    acc[7] = block_value<true>(sm_tab, b.w, h.w, X, acc[7]);
 }
 
 // Sums v[r] over the 32 lanes for r = 0..7 through the warp's shared-memory
@@ -589,12 +603,9 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
             LaneX X;
             load_lane_x(xq_p + (joint ? lane_col : uint32_t(cg * 32 + lane)) * uint32_t(kXqBytesPerCol),
                         !joint || lane_in, X);
-            float v[8];
-            record_values(sm_tab, a, b, h, X, v);
+            record_accumulate(sm_tab, a, b, h, X, acc);  // acc is zero when the joint pass begins
             pass_parity ^= 1;
             if (!joint) {
-#pragma unroll
-                for (int r = 0; r < 8; ++r) acc[r] += v[r];
                 if (++cg == CGf) {  // row group done: fold its eight accumulators into this lane's row
                     const float t = transpose_partial(red, lane, acc);
                     if (gi == 0) s0 = t; else if (gi == 1) s1 = t; else s2 = t;
@@ -608,7 +619,7 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
                 // k = l % 4, l % 4 + 4, ... of every row group's segment of the buffer
                 __syncwarp();
 #pragma unroll
-                for (int r = 0; r < 8; ++r) red[r * kRedStride + lane] = v[r];
+                for (int r = 0; r < 8; ++r) red[r * kRedStride + lane] = acc[r];
                 __syncwarp();
                 const float* rr = red + (lane >> 2) * kRedStride;
                 for (int k = lane & 3; k < rem; k += 4) {
