@@ -231,7 +231,7 @@ k_gemv_batched(const DeviceTables* __restrict__ tab, const unsigned char* __rest
                 int n2 = 0;
 #pragma unroll
                 for (int k = 0; k < 6; ++k) n2 = dp4a_ss(fb.y[k], fb.y[k], n2);
-                const float scale = lds32f(fb.goff | ((uint32_t(n2) >> 2) & 0x7Cu));  // gain[g] / sqrt(16 m)
+                const float scale = lds32f(fb.goff | (uint32_t(n2) & 0x1F0u));  // gain[g] / sqrt(16 m)
                 const int tile_id = (j % RB) * PC + 2 * (j / RB);  // + colsel
                 unsigned char* dst = tiles + (tile_id + colsel) * kTileBytes + row16 * kTileRow;
                 *reinterpret_cast<uint4*>(dst) = make_uint4(fb.y[0], fb.y[1], fb.y[2], fb.y[3]);

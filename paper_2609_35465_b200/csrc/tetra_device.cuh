@@ -139,8 +139,8 @@ __device__ __forceinline__ void file_to_device_word(uint64_t w, const DeviceTabl
 constexpr uint32_t kSmRows = 0;
 constexpr uint32_t kSmMid = 16384;
 constexpr uint32_t kSmScale = 24576;
-constexpr uint32_t kSmMaskH = 24832;
-constexpr uint32_t kSmMaskHr = 24896;
+constexpr uint32_t kSmMaskH = 25600;
+constexpr uint32_t kSmMaskHr = 25664;
 constexpr uint32_t kSmAlign = 16384;  // the staged copy starts on a 16 KiB boundary of shared memory
 static_assert(kSmMid == offsetof(DeviceTables, mid_fast) - kFastOffset, "staged layout");
 static_assert(kSmScale == offsetof(DeviceTables, scale) - kFastOffset, "staged layout");
@@ -172,7 +172,7 @@ constexpr uint32_t kRank4Step = 4u << 16;
 
 struct FastBlock {
     uint32_t y[6];  // the lattice point, int8 x 4, coordinate 4k+i in byte i of y[k]
-    uint32_t goff;  // shared-memory address of the gain's half of the scale table (bit 7 = g)
+    uint32_t goff;  // shared-memory address of the gain's half of the scale table (bit 9 = g)
 };
 
 // 1 if the 11-bit row index in the top bits of `x` lies in the last 32 slots of its class.
@@ -196,11 +196,11 @@ __device__ __forceinline__ void fast_decode(uint32_t sm_tab, uint32_t w0, uint32
     if (HI) {
         addr2 = ((w1pair >> 14) & 0x1FFCu) | (sm_tab + kSmMid);
         x4 = ((w1pair >> 25) & 0x3Cu) | (sm_tab + kSmMaskHr);
-        out.goff = ((w1pair >> 24) & 0x80u) | (sm_tab + kSmScale);
+        out.goff = ((w1pair >> 22) & 0x200u) | (sm_tab + kSmScale);
     } else {
         addr2 = ((w1pair << 2) & 0x1FFCu) | (sm_tab + kSmMid);
         x4 = ((w1pair >> 9) & 0x3Cu) | (sm_tab + kSmMaskHr);
-        out.goff = ((w1pair >> 8) & 0x80u) | (sm_tab + kSmScale);
+        out.goff = ((w1pair >> 6) & 0x200u) | (sm_tab + kSmScale);
     }
     const uint32_t row1 = lds32(addr1);
     const uint32_t row2 = lds32(addr2);

@@ -105,7 +105,7 @@ constexpr int kFastThreads = 512;
 constexpr int kFastWarps = kFastThreads / 32;
 constexpr int kRedStride = 36;                 // floats per row of the transpose buffer (32 + pad)
 constexpr int kRedFloats = 8 * kRedStride;     // per warp
-constexpr int kRowAccFloats = 2048;            // k_gemv_fast: per-CTA buffer of per-(column group, row) sums
+constexpr int kRowAccFloats = 1920;            // k_gemv_fast: per-CTA buffer of per-(column group, row) sums
 constexpr int kXqBytesPerCol = 80;             // 3 planes x 24 bytes, step, sum
 
 struct LaneX {
@@ -144,9 +144,9 @@ __device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint3
     }
     // |sum_j y_j q_j| <= sqrt(24 * 416) * 2^23 < 2^31: the block's dot product is an exact int32
     int dot = dh * 65536 + (dm * 256 + dl);
-    // n2 = 16 m; the scale table holds gain[g] / sqrt(16 m) at 128 g + 4 m.  The index is masked into
-    // the table, so the load stays aligned and in bounds whatever the inputs are.
-    const float scale = lds32f(fb.goff | ((uint32_t(n2) >> 2) & 0x7Cu));
+    // n2 = 16 m; the scale table holds gain[g] / sqrt(16 m) at 512 g + 16 m, so n2 is the byte offset.  It
+    // is masked into the table, so the load stays aligned and in bounds whatever the inputs are.
+    const float scale = lds32f(fb.goff | (uint32_t(n2) & 0x1F0u));
     return fmaf(float(dot), scale * X.step, addend);  // addend: the caller's running sum (one FFMA)
 }
 

@@ -238,7 +238,8 @@ int build_device_tables(DeviceTables* out, const float* gain2) {
         out->mask_hr[v] = mhr;
     }
     for (int g = 0; g < 2; ++g)
-        for (int m = 0; m < 32; ++m) out->scale[g][m] = out->gain[g] * out->paper.rsqrt16m[m];
+        for (int m = 0; m < 32; ++m)
+            for (int k = 0; k < 4; ++k) out->scale[g][m][k] = k == 0 ? out->gain[g] * out->paper.rsqrt16m[m] : 0.f;
     return 0;
 }
 

@@ -17,7 +17,7 @@ struct PaperTables {
 static_assert(sizeof(PaperTables) == 18816, "paper table blob is 18,816 bytes");
 
 constexpr uint32_t kTableMagic = 0x54455442u;  // "TETB"
-constexpr uint32_t kTableVersion = 5;
+constexpr uint32_t kTableVersion = 6;
 constexpr int kRank4Slots = 32;                // slots at the end of each class whose pool is patched
 constexpr int kMiddleClass0 = 1240;            // N0 of Sec. 3.3 (checked at build)
 
@@ -37,12 +37,13 @@ struct DeviceTables {
     //  sub-table's offset can be OR-ed into an index instead of added)
     uint32_t rows_fast[4096];   // +0
     uint32_t mid_fast[2048];    // +16384: rows_fast[mix(i2)], indexed by i2 directly
-    float scale[2][32];         // +24576: gain[g] / sqrt(16 m)
+    float scale[2][32][4];      // +24576: gain[g] / sqrt(16 m) in entry [g][m][0]: 16 bytes per m, so that the
+                                //         block's squared norm 16 m is the byte offset itself
     // Pattern-byte masks of the Turyn coordinates: bit 4j+2 set where the
     // Hamming word has coordinate j set; H for a and b, H' for x.
-    uint32_t mask_h[16];        // +24832
-    uint32_t mask_hr[16];       // +24896
-    uint32_t pad_[16];          // +24960 (spare)
+    uint32_t mask_h[16];        // +25600
+    uint32_t mask_hr[16];       // +25664
+    uint32_t pad_[16];          // +25728 (spare)
     // ---- pack-time only (global memory) ------------------------------------
     // 12 trellis bits (s8 | b1<<6 | b2<<7 | b3<<11) -> Turyn coordinates a | b<<4 | x<<8.
     uint16_t trellis_to_abx[4096];
