@@ -70,7 +70,7 @@ __device__ __forceinline__ void emit_block(const FastBlock& fb, int8_t* __restri
 #pragma unroll
     for (int k = 0; k < 6; ++k)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) y[4 * k + i] = int(int8_t((fb.y[k] >> (8 * i)) & 0xFF));
+        for (int i = 0; i < 4; ++i) y[4 * k + i] = -int(int8_t((fb.y[k] >> (8 * i)) & 0xFF));  // the decoder emits -y
     int norm = 0;
 #pragma unroll
     for (int k = 0; k < 24; ++k) norm += y[k] * y[k];

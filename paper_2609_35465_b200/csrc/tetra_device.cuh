@@ -6,12 +6,12 @@
 //     tetra_decode_blocks and by the paper-design GEMV.
 //   * the fast decoder: works on the re-ordered 48-bit device word written by
 //     tetra_pack_codes and on tables staged in shared memory.  It produces the
-//     lattice point as packed int8, four coordinates per register and one PRMT
-//     per four: a selector nibble is rank | c << 2 and the 8-byte PRMT pool holds
-//     the rank lists of Sec. 3.3 for the block's parity p.  Branch-free: rows
-//     with a coordinate of rank 4 sit in the last 32 slots of their class, and
-//     for those slots two multiply-adds turn the pool's rank-2 entries into the
-//     rank-4 values.
+//     lattice point (negated) as packed int8, four coordinates per register and
+//     one PRMT per four: a selector nibble is c | rank << 1 and the 8-byte PRMT
+//     pool holds the rank lists of Sec. 3.3 for the block's parity p.
+//     Branch-free: rows with a coordinate of rank 4 sit in the first 32 slots of
+//     their class, and for those slots one select swaps in a pool word whose
+//     rank-2 entries are the rank-4 values.
 #pragma once
 #include <cstdint>
 #include <cuda_fp16.h>
@@ -160,27 +160,25 @@ __device__ __forceinline__ unsigned char* stage_fast_tables(const DeviceTables* 
 }
 constexpr uint32_t kTableSmemBytes = uint32_t(kFastBytes) + kSmAlign;
 
-// PRMT pools, indexed by rank | c << 2 (ranks 0..3 of the lists of Sec. 3.3):
-//   p = 0:  c = 0: 0, 4, -4, 8     c = 1: 2, -2, 6, -6
-//   p = 1:  c = 0: 1, -3, 5, -7    c = 1: -1, 3, -5, 7
-// The rank-4 values differ from the rank-2 ones (entries 2 and 6, byte 2 of each
-// word) by 4 s and -4 s with s = 2p - 1:  -8, 10 for p = 0;  9, -9 for p = 1.  Adding
-// +-(4 << 16) to the two words never carries out of byte 2.
-constexpr uint32_t kPool0Lo = 0x08FC0400u, kPool0Hi = 0xFA06FE02u;
-constexpr uint32_t kPool1Lo = 0xF905FD01u, kPool1Hi = 0x07FB03FFu;
-constexpr uint32_t kRank4Step = 4u << 16;
+// PRMT pools.  A selector nibble is c | rank << 1 (c: the coordinate's pattern bit, ranks 0..3 of the
+// lists of Sec. 3.3), so the low pool word serves ranks 0 and 1 and the high word ranks 2 and 3:
+//   lo = { r0c0, r0c1, r1c0, r1c1 }    hi = { r2c0, r2c1, r3c0, r3c1 }
+// The pools hold MINUS the coordinate (the scale table holds minus the block scale, so products come
+// out with the right sign):
+//   p = 0:  y = 0, 2 | 4, -2 | -4, 6 | 8, -6        p = 1:  y = 1, -1 | -3, 3 | 5, -5 | -7, 7
+// A row with a coordinate of rank 4 (y = -8, 10 for p = 0; 9, -9 for p = 1) stores it as rank 2 and
+// sits in the first kRank4Slots slots of its class; for those slots the two rank-2 bytes of the high
+// word become the rank-4 values, which in this sign convention is the same XOR for both parities.
+constexpr uint32_t kPool0Lo = 0x02FCFE00u, kPool0Hi = 0x06F8FA04u;
+constexpr uint32_t kPool1Lo = 0xFD0301FFu, kPool1Hi = 0xF90705FBu;
+constexpr uint32_t kRank4Patch = 0x00000C0Cu;
+constexpr uint32_t kSpecialAddrMask = uint32_t(2048 - kRank4Slots) * 4u;  // zero <=> slot < kRank4Slots
+static_assert(kRank4Slots == 32 && kSpecialAddrMask == 0x1F80u, "special slots are the first 32 of a class");
 
 struct FastBlock {
-    uint32_t y[6];  // the lattice point, int8 x 4, coordinate 4k+i in byte i of y[k]
+    uint32_t y[6];  // MINUS the lattice point, int8 x 4, coordinate 4k+i in byte i of y[k]
     uint32_t goff;  // shared-memory address of the gain's half of the scale table (bit 9 = g)
 };
-
-// 1 if the 11-bit row index in the top bits of `x` lies in the last 32 slots of its class.
-__device__ __forceinline__ uint32_t top_slots_flag(uint32_t x) {
-    uint32_t f;
-    asm("{ .reg .u32 t; add.cc.u32 t, %1, %2; addc.u32 %0, 0, 0; }" : "=r"(f) : "r"(x), "r"(uint32_t(kRank4Slots) << 21));
-    return f;
-}
 
 // HI = false: w1 sits in bits 0..15 of `w1pair`; HI = true: in bits 16..31.
 // sm_tab: shared-memory address of the staged tables, a multiple of 16 KiB, so
@@ -214,22 +212,19 @@ __device__ __forceinline__ void fast_decode(uint32_t sm_tab, uint32_t w0, uint32
     const uint32_t sel1 = row1 ^ ma ^ mx;
     const uint32_t sel2 = row2 ^ mb ^ mx;
     const uint32_t sel3 = row3 ^ (ma ^ mb) ^ mx;
-    // p = r ^ q sits at bit 13 of both row addresses; 2^13 * 2^19 = 2^32 turns it into 0 / 1 on the
-    // multiplier pipe, and multiply-adds pick and patch the pools: the logic pipe sees one LOP3 of this
-    const uint32_t p = __umulhi((addr1 ^ addr3p) & 0x2000u, 0x80000u);
-    const uint32_t pool_lo = p * (kPool1Lo - kPool0Lo) + kPool0Lo;
-    const uint32_t pool_hi = p * (kPool1Hi - kPool0Hi) + kPool0Hi;
-    const uint32_t step = p * (2u * kRank4Step) - kRank4Step;  // (2p - 1) * (4 << 16)
-    const uint32_t f1 = top_slots_flag(w0 * 0x200000u);        // i1' in the top 11 bits
-    const uint32_t f3 = top_slots_flag(w0 * 0x200u);           // i3' in the top 11 bits
-    const uint32_t lo1 = f1 * step + pool_lo, hi1 = pool_hi - f1 * step;
-    const uint32_t lo3 = f3 * step + pool_lo, hi3 = pool_hi - f3 * step;
-    out.y[0] = prmt(lo1, hi1, sel1);
-    out.y[1] = prmt(lo1, hi1, sel1 >> 16);
-    out.y[2] = prmt(pool_lo, pool_hi, sel2);
-    out.y[3] = prmt(pool_lo, pool_hi, sel2 >> 16);
-    out.y[4] = prmt(lo3, hi3, sel3);
-    out.y[5] = prmt(lo3, hi3, sel3 >> 16);
+    // p = r ^ q sits at bit 13 of both row addresses: one test, two selects for the pools
+    const bool p = ((addr1 ^ addr3p) & 0x2000u) != 0;
+    const uint32_t lo = p ? kPool1Lo : kPool0Lo;
+    const uint32_t hi = p ? kPool1Hi : kPool0Hi;
+    const uint32_t hix = hi ^ kRank4Patch;
+    const uint32_t hi1 = (addr1 & kSpecialAddrMask) ? hi : hix;
+    const uint32_t hi3 = (addr3p & kSpecialAddrMask) ? hi : hix;
+    out.y[0] = prmt(lo, hi1, sel1);
+    out.y[1] = prmt(lo, hi1, sel1 >> 16);
+    out.y[2] = prmt(lo, hi, sel2);
+    out.y[3] = prmt(lo, hi, sel2 >> 16);
+    out.y[4] = prmt(lo, hi3, sel3);
+    out.y[5] = prmt(lo, hi3, sel3 >> 16);
 }
 
 // ---------------------------------------------------------------------------

@@ -134,7 +134,10 @@ __device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint3
                                              float addend = 0.f) {
     FastBlock fb;
     fast_decode<HI>(sm_tab, w0, w1pair, fb);
-    int dh = 0, dm = 0, dl = 0, n2 = 0;
+    // The squared norm 16 m is accumulated on top of the address of the gain's half of the scale table:
+    // that table holds -gain[g] / sqrt(16 m) at 512 g + 16 m, so the sum IS the address of the scale
+    // (16 m <= 416 for every word, Sec. 3.4, so it stays inside the table's half).
+    int dh = 0, dm = 0, dl = 0, n2 = int(fb.goff);
 #pragma unroll
     for (int k = 0; k < 6; ++k) {
         dh = dp4a_ss(fb.y[k], X.hi[k], dh);
@@ -143,10 +146,9 @@ __device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint3
         n2 = dp4a_ss(fb.y[k], fb.y[k], n2);
     }
     // |sum_j y_j q_j| <= sqrt(24 * 416) * 2^23 < 2^31: the block's dot product is an exact int32
+    // (of -y: the scale carries the other minus sign)
     int dot = dh * 65536 + (dm * 256 + dl);
-    // n2 = 16 m; the scale table holds gain[g] / sqrt(16 m) at 512 g + 16 m, so n2 is the byte offset.  It
-    // is masked into the table, so the load stays aligned and in bounds whatever the inputs are.
-    const float scale = lds32f(fb.goff | (uint32_t(n2) & 0x1F0u));
+    const float scale = lds32f(uint32_t(n2));
     return fmaf(float(dot), scale * X.step, addend);  // addend: the caller's running sum (one FFMA)
 }
 

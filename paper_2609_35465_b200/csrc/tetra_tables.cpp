@@ -170,9 +170,9 @@ int build_device_tables(DeviceTables* out, const float* gain2) {
     out->magic = kTableMagic;
     out->version = kTableVersion;
 
-    // Fast-path rows.  Per class: rows holding a rank-4 coordinate go to the last
+    // Fast-path rows.  Per class: rows holding a rank-4 coordinate go to the first
     // kRank4Slots slots, topped up with rows that use ranks 0 and 1 only (a patched
-    // pool serves ranks 0, 1 and 4); everything else keeps its order in front.
+    // pool serves ranks 0, 1 and 4); everything else keeps its order behind them.
     for (int cls = 0; cls < 2; ++cls) {
         std::vector<int> tail_rows, fillers, front;
         for (int i = 0; i < 2048; ++i) {
@@ -198,22 +198,25 @@ int build_device_tables(DeviceTables* out, const float* gain2) {
             }
         }
         if (int(tail_rows.size()) > kRank4Slots) return -25;
-        while (int(tail_rows.size()) < kRank4Slots) {
-            if (fillers.empty()) return -26;
-            tail_rows.push_back(fillers.back());
-            fillers.pop_back();
-        }
-        front.insert(front.end(), fillers.begin(), fillers.end());
+        // Fillers are taken cheapest first and go in front of the rank-4 rows, so slot 0 of class 0 is
+        // the all-zero row: the all-zero device word then decodes to the origin, which the kernels rely
+        // on when they pad.
+        const int nfill = kRank4Slots - int(tail_rows.size());
+        if (int(fillers.size()) < nfill) return -26;
+        std::vector<int> special(fillers.begin(), fillers.begin() + nfill);
+        special.insert(special.end(), tail_rows.begin(), tail_rows.end());
+        front.insert(front.end(), fillers.begin() + nfill, fillers.end());
         std::sort(front.begin(), front.end());
         if (int(front.size()) != 2048 - kRank4Slots) return -27;
+        if (cls == 0 && out->paper.rows[special[0]] != 0u) return -28;
         for (int slot = 0; slot < 2048; ++slot) {
-            const int i = slot < int(front.size()) ? front[slot] : tail_rows[slot - int(front.size())];
+            const int i = slot < kRank4Slots ? special[slot] : front[slot - kRank4Slots];
             const uint32_t row = out->paper.rows[2048 * cls + i];
             uint32_t fast = 0;
             for (int j = 0; j < 8; ++j) {
                 unsigned r = (row >> (4 * j)) & 15u;
                 if (r == 4) r = 2;
-                fast |= r << (4 * j);
+                fast |= (r << 1) << (4 * j);
             }
             out->rows_fast[2048 * cls + slot] = fast;
             out->row_perm[cls][i] = static_cast<uint16_t>(slot);
@@ -223,23 +226,27 @@ int build_device_tables(DeviceTables* out, const float* gain2) {
     for (int i2 = 0; i2 < 2048; ++i2) {
         const int idx = i2 < n0 ? i2 : 2048 + (i2 - n0);
         const uint32_t row = out->paper.rows[idx];
-        for (int j = 0; j < 8; ++j)
-            if (((row >> (4 * j)) & 15u) > 3) return -23;
-        out->mid_fast[i2] = row;
+        uint32_t fast = 0;
+        for (int j = 0; j < 8; ++j) {
+            const unsigned r = (row >> (4 * j)) & 15u;
+            if (r > 3) return -23;
+            fast |= (r << 1) << (4 * j);
+        }
+        out->mid_fast[i2] = fast;
     }
     for (unsigned v = 0; v < 16; ++v) {
         const uint8_t h = span4(turyn.h, v), hr = span4(turyn.hr, v);
         uint32_t mh = 0, mhr = 0;
         for (int j = 0; j < 8; ++j) {
-            mh |= uint32_t((h >> j) & 1) << (4 * j + 2);
-            mhr |= uint32_t((hr >> j) & 1) << (4 * j + 2);
+            mh |= uint32_t((h >> j) & 1) << (4 * j);
+            mhr |= uint32_t((hr >> j) & 1) << (4 * j);
         }
         out->mask_h[v] = mh;
         out->mask_hr[v] = mhr;
     }
     for (int g = 0; g < 2; ++g)
         for (int m = 0; m < 32; ++m)
-            for (int k = 0; k < 4; ++k) out->scale[g][m][k] = k == 0 ? out->gain[g] * out->paper.rsqrt16m[m] : 0.f;
+            for (int k = 0; k < 4; ++k) out->scale[g][m][k] = k == 0 ? -(out->gain[g] * out->paper.rsqrt16m[m]) : 0.f;
     return 0;
 }
 

@@ -17,8 +17,8 @@ struct PaperTables {
 static_assert(sizeof(PaperTables) == 18816, "paper table blob is 18,816 bytes");
 
 constexpr uint32_t kTableMagic = 0x54455442u;  // "TETB"
-constexpr uint32_t kTableVersion = 6;
-constexpr int kRank4Slots = 32;                // slots at the end of each class whose pool is patched
+constexpr uint32_t kTableVersion = 7;
+constexpr int kRank4Slots = 32;                // slots at the start of each class whose pool is patched
 constexpr int kMiddleClass0 = 1240;            // N0 of Sec. 3.3 (checked at build)
 
 // Everything tetra_build_table copies to the device, in one blob.
@@ -29,17 +29,19 @@ struct DeviceTables {
     uint32_t version;           // 18828
     // ---- fast path: everything below is staged in shared memory ------------
     // Rank rows for PRMT lookup, class by class in the permuted order of
-    // row_perm: nibble j = rank (0..3).  The last 32 slots of each class hold the
-    // rows with a coordinate of rank 4 (stored there as rank 2) and, as fillers,
-    // rows that use ranks 0 and 1 only: for those slots the kernels patch the
-    // rank-2 entries of the PRMT pool to the rank-4 values.
+    // row_perm: nibble j = rank << 1 (ranks 0..3; bit 0 is where the pattern bit
+    // goes).  The first 32 slots of each class hold the rows with a coordinate of
+    // rank 4 (stored there as rank 2) and, as fillers, rows that use ranks 0 and
+    // 1 only: for those slots the kernels swap in a PRMT pool word whose rank-2
+    // entries are the rank-4 values.
     // (the kernels place this part on a 16 KiB boundary of shared memory, so each
     //  sub-table's offset can be OR-ed into an index instead of added)
     uint32_t rows_fast[4096];   // +0
     uint32_t mid_fast[2048];    // +16384: rows_fast[mix(i2)], indexed by i2 directly
-    float scale[2][32][4];      // +24576: gain[g] / sqrt(16 m) in entry [g][m][0]: 16 bytes per m, so that the
-                                //         block's squared norm 16 m is the byte offset itself
-    // Pattern-byte masks of the Turyn coordinates: bit 4j+2 set where the
+    float scale[2][32][4];      // +24576: -gain[g] / sqrt(16 m) in entry [g][m][0]: 16 bytes per m, so that the
+                                //         block's squared norm 16 m is the byte offset itself (minus: the
+                                //         fast decoder emits -y)
+    // Pattern-byte masks of the Turyn coordinates: bit 4j set where the
     // Hamming word has coordinate j set; H for a and b, H' for x.
     uint32_t mask_h[16];        // +25600
     uint32_t mask_hr[16];       // +25664
