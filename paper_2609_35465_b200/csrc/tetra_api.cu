@@ -84,7 +84,7 @@ int tetra_build_table(void* table_dev, size_t bytes, const float* gain2_host, vo
         t->gain[0] = gain2_host[0];
         t->gain[1] = gain2_host[1];
         for (int g = 0; g < 2; ++g)
-            for (int m = 0; m < 32; ++m) t->scale[g][m][0] = -(t->gain[g] * t->paper.rsqrt16m[m]);
+            for (int m = 0; m < 32; ++m) t->scale[0][m][2 * g] = -(t->gain[g] * t->paper.rsqrt16m[m]);
     }
     cudaError_t e = cudaMemcpyAsync(table_dev, t, sizeof(DeviceTables), cudaMemcpyHostToDevice, as_stream(stream));
     if (e == cudaSuccess) e = cudaStreamSynchronize(as_stream(stream));

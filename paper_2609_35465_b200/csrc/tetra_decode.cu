@@ -81,7 +81,7 @@ __device__ __forceinline__ void emit_block(const FastBlock& fb, int8_t* __restri
                  (uint32_t(y[4 * k + 2] & 0xFF) << 16) | (uint32_t(y[4 * k + 3] & 0xFF) << 24);
     if (mg_out) {
         mg_out[2 * block] = uint8_t(norm >> 4);
-        mg_out[2 * block + 1] = uint8_t((fb.goff >> 9) & 1u);
+        mg_out[2 * block + 1] = uint8_t((fb.goff >> 3) & 1u);
     }
 }
 

@@ -177,7 +177,7 @@ static_assert(kRank4Slots == 32 && kSpecialAddrMask == 0x1F80u, "special slots a
 
 struct FastBlock {
     uint32_t y[6];  // MINUS the lattice point, int8 x 4, coordinate 4k+i in byte i of y[k]
-    uint32_t goff;  // shared-memory address of the gain's half of the scale table (bit 9 = g)
+    uint32_t goff;  // shared-memory address of the scale table plus 8 g (the gain's column of the table)
 };
 
 // HI = false: w1 sits in bits 0..15 of `w1pair`; HI = true: in bits 16..31.
@@ -194,11 +194,11 @@ __device__ __forceinline__ void fast_decode(uint32_t sm_tab, uint32_t w0, uint32
     if (HI) {
         addr2 = ((w1pair >> 14) & 0x1FFCu) | (sm_tab + kSmMid);
         x4 = ((w1pair >> 25) & 0x3Cu) | (sm_tab + kSmMaskHr);
-        out.goff = ((w1pair >> 22) & 0x200u) | (sm_tab + kSmScale);
+        out.goff = ((w1pair >> 28) & 8u) | (sm_tab + kSmScale);
     } else {
         addr2 = ((w1pair << 2) & 0x1FFCu) | (sm_tab + kSmMid);
         x4 = ((w1pair >> 9) & 0x3Cu) | (sm_tab + kSmMaskHr);
-        out.goff = ((w1pair >> 6) & 0x200u) | (sm_tab + kSmScale);
+        out.goff = ((w1pair >> 12) & 8u) | (sm_tab + kSmScale);
     }
     const uint32_t row1 = lds32(addr1);
     const uint32_t row2 = lds32(addr2);

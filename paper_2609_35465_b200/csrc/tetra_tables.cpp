@@ -246,7 +246,9 @@ int build_device_tables(DeviceTables* out, const float* gain2) {
     }
     for (int g = 0; g < 2; ++g)
         for (int m = 0; m < 32; ++m)
-            for (int k = 0; k < 4; ++k) out->scale[g][m][k] = k == 0 ? -(out->gain[g] * out->paper.rsqrt16m[m]) : 0.f;
+            for (int k = 0; k < 4; ++k) out->scale[g][m][k] = 0.f;
+    for (int g = 0; g < 2; ++g)
+        for (int m = 0; m < 32; ++m) out->scale[0][m][2 * g] = -(out->gain[g] * out->paper.rsqrt16m[m]);
     return 0;
 }
 

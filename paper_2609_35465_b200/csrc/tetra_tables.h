@@ -38,9 +38,11 @@ struct DeviceTables {
     //  sub-table's offset can be OR-ed into an index instead of added)
     uint32_t rows_fast[4096];   // +0
     uint32_t mid_fast[2048];    // +16384: rows_fast[mix(i2)], indexed by i2 directly
-    float scale[2][32][4];      // +24576: -gain[g] / sqrt(16 m) in entry [g][m][0]: 16 bytes per m, so that the
-                                //         block's squared norm 16 m is the byte offset itself (minus: the
-                                //         fast decoder emits -y)
+    float scale[2][32][4];      // +24576: -gain[g] / sqrt(16 m) in entry [0][m][2 g] (the second half is spare):
+                                //         16 bytes per m, so that the block's squared norm 16 m is the byte
+                                //         offset itself, and the two gains 8 bytes apart, so that lanes with
+                                //         nearby m or different g read different banks.  Minus: the fast
+                                //         decoder emits -y.
     // Pattern-byte masks of the Turyn coordinates: bit 4j set where the
     // Hamming word has coordinate j set; H for a and b, H' for x.
     uint32_t mask_h[16];        // +25600
