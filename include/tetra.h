@@ -48,7 +48,8 @@ enum {
     TETRA_WORD_BYTES = 6,
     TETRA_MAX_BATCH = 16,
     TETRA_PAPER_TABLE_BYTES = 18816, /* 16384 + 2304 + 128, Sec. 3.4 */
-    TETRA_NOALLOC_MAX_K = 24576      /* largest K tetra_gemv_noalloc accepts */
+    TETRA_NOALLOC_MAX_K = 24576,     /* largest K tetra_gemv_noalloc accepts */
+    TETRA_LIST_MAX = 8               /* most matrices in one tetra_gemv_list call */
 };
 
 /* Human-readable name of a status code (static storage). */
@@ -106,7 +107,19 @@ int tetra_decode_packed(const void *packed_dev, const void *table_dev, int8_t *y
  * codes: packed layout of an N x ceil(K/24) matrix (16-byte aligned).
  * row_scales: float32 [N].  x: float16 [batch][K] (2-byte aligned; 16-byte
  * aligned rows are faster).  y: float32 [batch][N], fully overwritten.
- * Products are exact and accumulation is float32.  1 <= batch <= 16. */
+ * 1 <= batch <= 16.
+ * Arithmetic: the 24 activations of a block column are held as 24-bit fixed
+ * point with a power-of-two step 2^(E-22), 2^E <= max |x_j| < 2^(E+1) over the
+ * column; the products with the lattice coordinates and their sum over the
+ * block are exact integers, converted once and accumulated in float32 across
+ * blocks.  An activation is therefore represented exactly when |x_j| >=
+ * 2^(E-12), i.e. within a factor 4096 of its column's largest; a smaller one is
+ * rounded to a multiple of the step (at most 2^-23 of the column's largest).
+ * Non-finite activations: if any of a block column's 24 activations is NaN or
+ * infinite, every output row comes out NaN (every row reads every column); a
+ * non-finite value in the unquantized tail propagates by the IEEE rules of
+ * float32 multiply-add.  The same holds for every decode-and-multiply entry
+ * point below except tetra_gemv_paper_design, which multiplies in float32. */
 int tetra_gemv(const void *codes, const float *row_scales, const void *table,
                const void *x, float *y, int N, int K, int batch, void *stream);
 
@@ -130,6 +143,18 @@ typedef struct {
     int32_t K;
 } tetra_problem;
 
+/* Batch-1 products of a SHORT list of independent matrices (1 <= count <=
+ * TETRA_LIST_MAX) in one kernel launch, with no scratch memory and nothing to
+ * plan: the call for the matrices of one dependency step of a model (q, k and v
+ * of a layer; gate and up), the unit Sec. 5.2 times ("one launch per matrix").
+ * The descriptors are read before the call returns.  Everything that does not
+ * depend on the activations (decode tables, first code words, row scales) is
+ * started before the kernel waits for its predecessor in the stream, so a chain
+ * of such calls overlaps each launch's set-up with the previous launch.
+ * tetra_gemv and tetra_gemv_tail are this call with one matrix. */
+int tetra_gemv_list(const tetra_problem *problems_host, int count, const void *table,
+                    void *stream);
+
 /* Batch-1 products of a list of independent matrices from one persistent grid
  * (the tables staged in shared memory once, every warp walking independent
  * eight-row units of the whole list).  The list is planned once and run many
@@ -142,7 +167,13 @@ typedef struct {
  *                                  then the persistent kernel computes every y.
  * workspace_dev: 16-byte aligned device memory owned by the caller; it belongs to
  * the plan until the last run using it has completed, and runs that share a
- * workspace must not overlap on the GPU.  tetra_gemv_grouped = plan + run. */
+ * workspace must not overlap on the GPU.  The plan in the workspace describes
+ * itself (list, mode, index arrays): a planned workspace may be copied to other
+ * device memory and run from there, on the device it was planned for.
+ * tetra_gemv_grouped_plan copies from host memory it frees before returning:
+ * call it outside stream capture (tetra_gemv_grouped_run may be captured).
+ * tetra_gemv_grouped = plan + run.  Lists of at most TETRA_LIST_MAX matrices are
+ * served faster by tetra_gemv_list. */
 size_t tetra_grouped_workspace_bytes(const tetra_problem *problems_host, int count);
 int tetra_gemv_grouped_plan(const tetra_problem *problems_host, int count, void *workspace_dev,
                             size_t workspace_bytes, void *stream);
@@ -224,7 +255,11 @@ int tetra_gemv_grouped_hostio(void *workspace_dev, const void *table, const void
  *     Nothing in it needs clearing (each call rewrites all it reads), but two
  *     calls that run on the GPU at the same time, on any streams, race on it:
  *     keep calls on one device in stream order, or serialise them.
- *   - Enqueues one small copy and two kernels on `stream`; does not synchronise. */
+ *   - K < 24 with a tail (no whole word in a row) returns TETRA_ERR_SHAPE, as in
+ *     tetra_gemv_tail.
+ *   - Enqueues three kernels on `stream` (the first writes the product's
+ *     description into the array from its own parameters, so no host memory is
+ *     referenced after the call returns); does not synchronise. */
 int tetra_gemv_noalloc(const void *codes, const float *row_scales, const void *table,
                        const void *x, float *y, int N, int K, const void *tail, void *stream);
 

@@ -129,8 +129,14 @@ int tetra_gemv_tail(const void* codes, const float* row_scales, const void* tabl
     const bool tail_mode = tail != nullptr || K % 24 == 0;
     const int B = tail_mode ? K / 24 : (K + 23) / 24;
     if (B <= 0 || B > kMaxBlocksPerRow) return TETRA_ERR_SHAPE;
-    Problem p{codes, row_scales, x, (K % 24) ? tail : nullptr, y, N, K};
-    return cuda_status(launch_gemv_fast(p, batch, B, table, as_stream(stream)));
+    ListDesc list{};
+    list.count = 1;
+    list.total_groups = (N + 7) / 8;
+    list.group_prefix[0] = 0;
+    list.group_prefix[1] = list.total_groups;
+    list.max_blocks = B;
+    list.problems[0] = Problem{codes, row_scales, x, (K % 24) ? tail : nullptr, y, N, K};
+    return cuda_status(launch_gemv_list(list, batch, table, as_stream(stream)));
 }
 
 int tetra_gemv(const void* codes, const float* row_scales, const void* table, const void* x, float* y, int N, int K,
@@ -153,6 +159,29 @@ static int check_problems(const tetra_problem* problems_host, int count) {
         if (B <= 0 || B > kMaxBlocksPerRow) return TETRA_ERR_SHAPE;
     }
     return TETRA_OK;
+}
+
+int tetra_gemv_list(const tetra_problem* problems_host, int count, const void* table, void* stream) {
+    if (!table) return TETRA_ERR_NULL;
+    if (!aligned(table, 16)) return TETRA_ERR_ALIGN;
+    const int rc = check_problems(problems_host, count);
+    if (rc) return rc;
+    if (count > TETRA_LIST_MAX) return TETRA_ERR_SHAPE;
+    ListDesc list{};
+    list.count = count;
+    long long groups = 0;
+    for (int i = 0; i < count; ++i) {
+        const tetra_problem& q = problems_host[i];
+        list.group_prefix[i] = int32_t(groups);
+        groups += (q.N + 7) / 8;
+        const int B = (q.tail || q.K % 24 == 0) ? q.K / 24 : (q.K + 23) / 24;
+        if (B > list.max_blocks) list.max_blocks = B;
+        list.problems[i] = Problem{q.codes, q.row_scales, q.x, (q.K % 24) ? q.tail : nullptr, q.y, q.N, q.K};
+    }
+    if (groups > 0x7FFFFFF0LL) return TETRA_ERR_SHAPE;
+    for (int i = count; i <= kListMax; ++i) list.group_prefix[i] = int32_t(groups);
+    list.total_groups = int32_t(groups);
+    return cuda_status(launch_gemv_list(list, 1, table, as_stream(stream)));
 }
 
 size_t tetra_grouped_workspace_bytes(const tetra_problem* problems_host, int count) {

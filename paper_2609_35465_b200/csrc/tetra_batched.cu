@@ -68,14 +68,17 @@ __device__ __forceinline__ void image_load(const __half* __restrict__ x, int K, 
 }
 // group_base: shared-memory address of the column's 1 KiB group for the vector's group of eight.
 __device__ __forceinline__ void image_store(const ImageTask& T, uint32_t group_base, int vec, int t) {
-    float mx = 0.f;
+    // largest magnitude as a bit pattern (a NaN or an infinity then counts as the largest)
+    uint32_t mxb = 0u;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) mx = fmaxf(mx, fabsf(T.v[i]));
-    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
-    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
-    const uint32_t e = __float_as_uint(mx) >> 23;  // biased exponent of the largest (finite float16 input)
-    const float step = mx > 0.f ? __uint_as_float((e - 22u) << 23) : 0.f;
-    const float inv = mx > 0.f ? __uint_as_float((276u - e) << 23) : 0.f;
+    for (int i = 0; i < 8; ++i) mxb = max(mxb, __float_as_uint(T.v[i]) & 0x7FFFFFFFu);
+    mxb = max(mxb, __shfl_xor_sync(0xFFFFFFFFu, mxb, 1));
+    mxb = max(mxb, __shfl_xor_sync(0xFFFFFFFFu, mxb, 2));
+    const bool finite = mxb < 0x7F800000u;
+    const uint32_t e = mxb >> 23;  // biased exponent of the largest
+    // a NaN or an infinity in the column makes its step NaN: every row that reads the column comes out NaN
+    const float step = !finite ? __uint_as_float(0x7FC00000u) : (mxb ? __uint_as_float((e - 22u) << 23) : 0.f);
+    const float inv = (finite && mxb) ? __uint_as_float((276u - e) << 23) : 0.f;
     uint32_t b[3][2];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {

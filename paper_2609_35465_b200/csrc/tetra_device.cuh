@@ -158,6 +158,16 @@ __device__ __forceinline__ unsigned char* stage_fast_tables(const DeviceTables* 
     for (uint32_t i = threadIdx.x; i < kFastBytes / 16; i += blockDim.x) dst[i] = src[i];
     return base;
 }
+// The same copy with cp.async (16 bytes per request, all of a thread's requests in flight at once);
+// the caller commits and waits for the group and synchronises the CTA before the tables are read.
+__device__ __forceinline__ unsigned char* stage_fast_tables_async(const DeviceTables* tab, unsigned char* smem) {
+    const uint32_t s = smem_u32(smem);
+    const uint32_t pad = ((s + kSmAlign - 1) & ~(kSmAlign - 1)) - s;
+    const char* src = reinterpret_cast<const char*>(tab) + kFastOffset;
+    for (uint32_t i = threadIdx.x; i < kFastBytes / 16; i += blockDim.x)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(s + pad + 16u * i), "l"(src + 16u * i));
+    return smem + pad;
+}
 constexpr uint32_t kTableSmemBytes = uint32_t(kFastBytes) + kSmAlign;
 
 // PRMT pools.  A selector nibble is c | rank << 1 (c: the coordinate's pattern bit, ranks 0..3 of the
@@ -235,7 +245,8 @@ __device__ __forceinline__ void fast_decode(uint32_t sm_tab, uint32_t w0, uint32
 // stored as three byte planes (bits 23..16 signed, 15..8 and 7..0 unsigned), four
 // coordinates per 32-bit word: words 0..5 high, 6..11 middle, 12..17 low plane;
 // word 18 = step (float), word 19 = sum(q_j).  A float16 x_j is held exactly when
-// |x_j| >= 2^(E-12); smaller ones are rounded to a multiple of the step.
+// |x_j| >= 2^(E-12); smaller ones are rounded to a multiple of the step.  If a value
+// is NaN or infinite the step is NaN (and the planes zero).
 __device__ __forceinline__ void quantise_column(const __half* __restrict__ x, int K, int c, uint32_t out[20]) {
     float v[24];
     const int k0 = 24 * c;
@@ -256,12 +267,17 @@ __device__ __forceinline__ void quantise_column(const __half* __restrict__ x, in
 #pragma unroll
         for (int j = 0; j < 24; ++j) v[j] = k0 + j < K ? __half2float(x[k0 + j]) : 0.f;
     }
-    float mx = 0.f;
+    // largest magnitude, compared as bit patterns (same order as the values for non-negative floats):
+    // a NaN or an infinity, whose exponent field is all ones, then counts as the largest
+    uint32_t mxb = 0u;
 #pragma unroll
-    for (int j = 0; j < 24; ++j) mx = fmaxf(mx, fabsf(v[j]));
-    const uint32_t e = __float_as_uint(mx) >> 23;  // biased exponent of the largest (finite float16 input)
-    const float step = mx > 0.f ? __uint_as_float((e - 22u) << 23) : 0.f;
-    const float inv = mx > 0.f ? __uint_as_float((276u - e) << 23) : 0.f;
+    for (int j = 0; j < 24; ++j) mxb = max(mxb, __float_as_uint(v[j]) & 0x7FFFFFFFu);
+    const bool finite = mxb < 0x7F800000u;
+    const uint32_t e = mxb >> 23;  // biased exponent of the largest
+    // A NaN or an infinity among the 24 values makes the step NaN, so every product with this column, and
+    // with it every output row that reads the column, comes out NaN instead of a finite, wrong number.
+    const float step = !finite ? __uint_as_float(0x7FC00000u) : (mxb ? __uint_as_float((e - 22u) << 23) : 0.f);
+    const float inv = (finite && mxb) ? __uint_as_float((276u - e) << 23) : 0.f;
     int sum = 0;
 #pragma unroll
     for (int k = 0; k < 6; ++k) {

@@ -4,8 +4,7 @@
 //                 per output row, a lane per block, the six table loads of
 //                 Fig. "decode", FP32 multiply-accumulate, shuffle reduction.
 //                 Kept as a comparison arm and cross-check.
-//   k_gemv_fast / k_gemv_units
-//                 the B200 design: a lane owns one block column and keeps its
+//   k_gemv_units  the B200 design (also in k_gemv_list, tetra_list.cu): a lane owns one block column and keeps its
 //                 24 activations in registers as 24-bit fixed point (three int8
 //                 planes, power-of-two step per block column, so float16 inputs
 //                 within 2^12 of the column's largest are held exactly); it
@@ -15,8 +14,6 @@
 //                 becomes a float, FP32 accumulation across blocks.  The ALU
 //                 pipe only unpacks fields; the integer-MAD pipe does the
 //                 arithmetic.
-//                 k_gemv_fast serves one matrix per launch and needs no
-//                 scratch memory (every CTA quantises x for itself).
 //                 k_gemv_units serves a planned list of matrices from one
 //                 persistent grid: k_prepare_x first writes the fixed-point
 //                 activations of every matrix to the plan's scratch area, then
@@ -27,12 +24,28 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
-#include <unordered_map>
 
-#include "tetra_device.cuh"
-#include "tetra_launch.h"
+#include "tetra_gemv_common.cuh"
 
 namespace tetra {
+
+cudaError_t device_sms(int* sms) {
+    static std::mutex mu;
+    static int cached[64] = {0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[dev] == 0) {
+        int n = 0;
+        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        cached[dev] = n;
+    }
+    *sms = cached[dev];
+    return cudaSuccess;
+}
 
 // ===========================================================================
 // Paper-design kernel
@@ -96,261 +109,6 @@ cudaError_t launch_gemv_paper(const void* codes, size_t row_stride, const float*
                                       static_cast<const DeviceTables*>(table), static_cast<const __half*>(x), y, N, K,
                                       B, ntail, static_cast<const __half*>(tail));
     return cudaGetLastError();
-}
-
-// ===========================================================================
-// Fast kernels: shared pieces
-// ===========================================================================
-constexpr int kFastThreads = 512;
-constexpr int kFastWarps = kFastThreads / 32;
-constexpr int kRedStride = 36;                 // floats per row of the transpose buffer (32 + pad)
-constexpr int kRedFloats = 8 * kRedStride;     // per warp
-constexpr int kRowAccFloats = 1920;            // k_gemv_fast: per-CTA buffer of per-(column group, row) sums
-constexpr int kXqBytesPerCol = 80;             // 3 planes x 24 bytes, step, sum
-
-struct LaneX {
-    uint32_t hi[6];   // bits 23..16 of q (signed), int8 x 4
-    uint32_t mid[6];  // bits 15..8 (unsigned)
-    uint32_t lo[6];   // bits 7..0 (unsigned)
-    float step;       // 2^(E-22)
-    int sum;          // sum of q over the 24 coordinates (kept in the record; unused by the kernels)
-};
-
-__device__ __forceinline__ void lane_x_from_words(const uint32_t q[20], bool active, LaneX& X) {
-#pragma unroll
-    for (int k = 0; k < 6; ++k) {
-        X.hi[k] = active ? q[k] : 0u;
-        X.mid[k] = active ? q[6 + k] : 0u;
-        X.lo[k] = active ? q[12 + k] : 0u;
-    }
-    X.step = active ? __uint_as_float(q[18]) : 0.f;
-    X.sum = active ? int(q[19]) : 0;
-}
-
-// One block: device word -> contribution scale_b * sum_j y_j x_j (Eq. (2) without
-// the row scale).
-template <bool HI>
-__device__ __forceinline__ float block_value(uint32_t sm_tab, uint32_t w0, uint32_t w1pair, const LaneX& X,
-                                             float addend = 0.f) {
-    FastBlock fb;
-    fast_decode<HI>(sm_tab, w0, w1pair, fb);
-    // The squared norm 16 m is accumulated on top of the address of the gain's half of the scale table:
-    // that table holds -gain[g] / sqrt(16 m) at 512 g + 16 m, so the sum IS the address of the scale
-    // (16 m <= 416 for every word, Sec. 3.4, so it stays inside the table's half).
-    int dh = 0, dm = 0, dl = 0, n2 = int(fb.goff);
-#pragma unroll
-    for (int k = 0; k < 6; ++k) {
-        dh = dp4a_ss(fb.y[k], X.hi[k], dh);
-        dm = dp4a_su(fb.y[k], X.mid[k], dm);
-        dl = dp4a_su(fb.y[k], X.lo[k], dl);
-        n2 = dp4a_ss(fb.y[k], fb.y[k], n2);
-    }
-    // |sum_j y_j q_j| <= sqrt(24 * 416) * 2^23 < 2^31: the block's dot product is an exact int32
-    // (of -y: the scale carries the other minus sign)
-    int dot = dh * 65536 + (dm * 256 + dl);
-    const float scale = lds32f(uint32_t(n2));
-    return fmaf(float(dot), scale * X.step, addend);  // addend: the caller's running sum (one FFMA)
-}
-
-// The eight blocks of one 48-byte record (rows 8G..8G+7 of one column).
-__device__ __forceinline__ void record_values(uint32_t sm_tab, const uint4& a, const uint4& b, const uint4& h,
-                                              const LaneX& X, float v[8]) {
-    v[0] = block_value<false>(sm_tab, a.x, h.x, X);
-    v[1] = block_value<true>(sm_tab, a.y, h.x, X);
-    v[2] = block_value<false>(sm_tab, a.z, h.y, X);
-    v[3] = block_value<true>(sm_tab, a.w, h.y, X);
-    v[4] = block_value<false>(sm_tab, b.x, h.z, X);
-    v[5] = block_value<true>(sm_tab, b.y, h.z, X);
-    v[6] = block_value<false>(sm_tab, b.z, h.w, X);
-    v[7] = block_value<true>(sm_tab, b.w, h.w, X);
-}
-
-// The same, added to the caller's eight running sums.
-__device__ __forceinline__ void record_accumulate(uint32_t sm_tab, const uint4& a, const uint4& b, const uint4& h,
-                                                  const LaneX& X, float acc[8]) {
-    acc[0] = block_value<false>(sm_tab, a.x, h.x, X, acc[0]);
-    acc[1] = block_value<true>(sm_tab, a.y, h.x, X, acc[1]);
-    acc[2] = block_value<false>(sm_tab, a.z, h.y, X, acc[2]);
-    acc[3] = block_value<true>(sm_tab, a.w, h.y, X, acc[3]);
-    acc[4] = block_value<false>(sm_tab, b.x, h.z, X, acc[4]);
-    acc[5] = block_value<true>(sm_tab, b.y, h.z, X, acc[5]);
-    acc[6] = block_value<false>(sm_tab, b.z, h.w, X, acc[6]);
-    acc[7] = block_value<true>(sm_tab, b.w, h.w, X, acc[7]);
-}
-
-// Sums v[r] over the 32 lanes for r = 0..7 through the warp's shared-memory
-// buffer.  Afterwards lane l holds, for row l / 4, the partial sum over lanes
-// 8 (l % 4) .. 8 (l % 4) + 7; the caller finishes with two shuffles.
-__device__ __forceinline__ float transpose_partial(float* red, int lane, const float v[8]) {
-    __syncwarp();
-#pragma unroll
-    for (int r = 0; r < 8; ++r) red[r * kRedStride + lane] = v[r];
-    __syncwarp();
-    const float4 s0 = *reinterpret_cast<const float4*>(red + (lane >> 2) * kRedStride + 8 * (lane & 3));
-    const float4 s1 = *reinterpret_cast<const float4*>(red + (lane >> 2) * kRedStride + 8 * (lane & 3) + 4);
-    return ((s0.x + s0.y) + (s0.z + s0.w)) + ((s1.x + s1.y) + (s1.z + s1.w));
-}
-
-// ===========================================================================
-// k_gemv_fast: one matrix per launch, no scratch memory
-// ===========================================================================
-struct FastSmemLayout {
-    uint32_t xq, red, rowacc, total;  // offsets from the 16 KiB-aligned table copy
-};
-__host__ __device__ inline FastSmemLayout fast_smem_layout(int max_blocks) {
-    FastSmemLayout L;
-    L.xq = uint32_t(kFastBytes);
-    L.red = L.xq + uint32_t(max_blocks) * kXqBytesPerCol;
-    L.rowacc = L.red + kFastWarps * kRedFloats * 4;
-    L.total = L.rowacc + kRowAccFloats * 4 + kSmAlign;
-    return L;
-}
-
-__global__ void __launch_bounds__(kFastThreads, 1)
-k_gemv_fast(const DeviceTables* __restrict__ tab, const Problem single, int batch, int max_blocks) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    pdl_release();
-    const FastSmemLayout L = fast_smem_layout(max_blocks);
-    unsigned char* smem = stage_fast_tables(tab, smem_raw);
-    pdl_wait();  // x may come from the previous kernel of the stream; the tables above do not
-    const uint32_t sm_tab = smem_u32(smem);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float* red = reinterpret_cast<float*>(smem + L.red) + warp * kRedFloats;
-    float* rowacc = reinterpret_cast<float*>(smem + L.rowacc);
-
-    for (int job = 0; job < batch; ++job) {  // batch column `job`
-        Problem P = single;
-        P.x = static_cast<const __half*>(P.x) + size_t(job) * P.K;
-        P.y = P.y + size_t(job) * P.N;
-        const int ntail = P.tail ? P.K % 24 : 0;
-        const int B = P.tail ? P.K / 24 : (P.K + 23) / 24;
-        const int groups = (P.N + 7) / 8;
-        const int g_begin = int((long long)blockIdx.x * groups / gridDim.x);
-        const int g_end = int((long long)(blockIdx.x + 1) * groups / gridDim.x);
-        const int CG = (B + 31) / 32;
-        __syncthreads();  // previous column's epilogue is done with xq / rowacc; tables are staged
-        for (int c = threadIdx.x; c < B; c += blockDim.x) {
-            uint32_t q[20];
-            quantise_column(static_cast<const __half*>(P.x), P.K, c, q);
-            uint4* dst = reinterpret_cast<uint4*>(smem + L.xq + c * kXqBytesPerCol);
-#pragma unroll
-            for (int k = 0; k < 5; ++k) dst[k] = make_uint4(q[4 * k], q[4 * k + 1], q[4 * k + 2], q[4 * k + 3]);
-        }
-        __syncthreads();
-
-        const bool narrow = CG <= kFastWarps;
-        const int RL = narrow ? kFastWarps / CG : 1;  // warps sharing a column group walk different rows
-        const int rl = narrow ? warp / CG : 0;
-        const int cg_step = narrow ? CG : kFastWarps;
-        // rows of this CTA are processed in chunks whose per-(column group, row) sums fit the buffer
-        const int chunk_groups = max(1, kRowAccFloats / (8 * CG));
-        const uint4* codes = static_cast<const uint4*>(P.codes);
-
-        for (int c_begin = g_begin; c_begin < g_end; c_begin += chunk_groups) {
-            const int c_end = min(g_end, c_begin + chunk_groups);
-            const int rows_chunk = (c_end - c_begin) * 8;
-            if (rl < RL) {
-                for (int cg = narrow ? warp % CG : warp; cg < CG; cg += cg_step) {
-                    const int col = cg * 32 + lane;
-                    const bool active = col < B;
-                    const unsigned char* xq_rec = smem + L.xq + (active ? col : 0) * kXqBytesPerCol;
-                    LaneX X;
-                    {
-                        uint32_t q[20];
-                        const uint4* src = reinterpret_cast<const uint4*>(xq_rec);
-#pragma unroll
-                        for (int k = 0; k < 5; ++k) {
-                            const uint4 u = src[k];
-                            q[4 * k] = u.x; q[4 * k + 1] = u.y; q[4 * k + 2] = u.z; q[4 * k + 3] = u.w;
-                        }
-                        lane_x_from_words(q, active, X);
-                    }
-                    const uint4 zero4 = make_uint4(0, 0, 0, 0);
-                    int g = c_begin + rl;
-                    uint4 n0 = zero4, n1 = zero4, n2 = zero4;
-                    if (g < c_end && active) {
-                        const uint4* rec = codes + size_t(g) * 3 * B + col;
-                        n0 = __ldg(rec); n1 = __ldg(rec + B); n2 = __ldg(rec + 2 * size_t(B));
-                    }
-                    for (; g < c_end; g += RL) {
-                        const uint4 a = n0, b = n1, h = n2;
-                        if (g + RL < c_end && active) {  // prefetch the next record
-                            const uint4* rec = codes + size_t(g + RL) * 3 * B + col;
-                            n0 = __ldg(rec); n1 = __ldg(rec + B); n2 = __ldg(rec + 2 * size_t(B));
-                        }
-                        float v[8];
-                        record_values(sm_tab, a, b, h, X, v);
-                        float sum = transpose_partial(red, lane, v);
-                        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
-                        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
-                        if ((lane & 3) == 0) rowacc[cg * rows_chunk + (g - c_begin) * 8 + (lane >> 2)] = sum;
-                    }
-                }
-            }
-            __syncthreads();
-            // epilogue: sum the column groups in a fixed order, row scale, tail (Sec. 5.1)
-            for (int t = threadIdx.x; t < rows_chunk; t += blockDim.x) {
-                const int row = c_begin * 8 + t;
-                if (row >= P.N) continue;
-                float acc = 0.f;
-                for (int cg = 0; cg < CG; ++cg) acc += rowacc[cg * rows_chunk + t];
-                float res = P.row_scales[row] * acc;
-                const __half* xh = static_cast<const __half*>(P.x);
-                const __half* tl = static_cast<const __half*>(P.tail);
-                for (int k = 0; k < ntail; ++k)
-                    res = fmaf(__half2float(tl[size_t(row) * ntail + k]), __half2float(xh[24 * B + k]), res);
-                P.y[row] = res;
-            }
-            __syncthreads();
-        }
-    }
-}
-
-// Launch with programmatic stream serialization allowed: the kernel may start while its predecessor
-// in the stream is still running and synchronises with it through pdl_wait().
-template <typename... KArgs, typename... Args>
-static cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t s, Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(unsigned(grid));
-    cfg.blockDim = dim3(unsigned(block));
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
-}
-
-static cudaError_t device_sms(int* sms) {
-    static int cached[64] = {0};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (cached[dev] == 0) {
-        int n = 0;
-        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(k_gemv_fast, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) return e;
-        cached[dev] = n;
-    }
-    *sms = cached[dev];
-    return cudaSuccess;
-}
-
-cudaError_t launch_gemv_fast(const Problem& single, int batch, int max_blocks, const void* table, cudaStream_t s) {
-    int sms = 0;
-    cudaError_t e = device_sms(&sms);
-    if (e != cudaSuccess) return e;
-    const FastSmemLayout L = fast_smem_layout(max_blocks);
-    if (L.total > 227u * 1024u) return cudaErrorInvalidValue;
-    const int groups = (single.N + 7) / 8;
-    const int grid = groups < sms ? groups : sms;
-    return launch_pdl(k_gemv_fast, grid, kFastThreads, L.total, s, static_cast<const DeviceTables*>(table), single,
-                      batch, max_blocks);
 }
 
 // ===========================================================================
@@ -489,17 +247,10 @@ __device__ __forceinline__ void load_lane_x(const unsigned char* xq_rec, bool ac
 constexpr int kUnitThreads = TETRA_UNIT_THREADS;
 constexpr int kUnitWarps = kUnitThreads / 32;
 
-__global__ void __launch_bounds__(kUnitThreads, 1)
-k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restrict__ ws) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    pdl_release();
-    unsigned char* smem = stage_fast_tables(tab, smem_raw);
-    const uint32_t sm_tab = smem_u32(smem);
+// Coarse mode: every warp walks its range of units (up to three row groups of one matrix, all columns).
+__device__ __forceinline__ void units_coarse(const unsigned char* __restrict__ ws, unsigned char* smem, uint32_t sm_tab) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float* red = reinterpret_cast<float*>(smem + kFastBytes) + warp * kRedFloats;
-    __syncthreads();  // the only CTA-wide barrier: tables are staged
-    pdl_wait();       // the plan's activation records come from k_prepare_x
-
     const PlanHeader* H = reinterpret_cast<const PlanHeader*>(ws);
     const Problem* problems = reinterpret_cast<const Problem*>(ws + H->off_problems);
     const int32_t* unit_prefix = reinterpret_cast<const int32_t*>(ws + H->off_unit_prefix);
@@ -658,17 +409,9 @@ k_gemv_units(const DeviceTables* __restrict__ tab, const unsigned char* __restri
 // Each unit leaves eight partial row sums in the scratch area and bumps its row group's counter; the
 // unit that finds all the other slices done adds them up in slice order (fixed order, no waiting,
 // no floating-point atomics), applies the row scale and the tail, and stores.
-__global__ void __launch_bounds__(kUnitThreads, 1)
-k_gemv_units_fine(const DeviceTables* __restrict__ tab, unsigned char* __restrict__ ws) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    pdl_release();
-    unsigned char* smem = stage_fast_tables(tab, smem_raw);
-    const uint32_t sm_tab = smem_u32(smem);
+__device__ __forceinline__ void units_fine(unsigned char* __restrict__ ws, unsigned char* smem, uint32_t sm_tab) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float* red = reinterpret_cast<float*>(smem + kFastBytes) + warp * kRedFloats;
-    __syncthreads();
-    pdl_wait();  // the plan's activation records and zeroed counters come from k_prepare_x
-
     const PlanHeader* H = reinterpret_cast<const PlanHeader*>(ws);
     const Problem* problems = reinterpret_cast<const Problem*>(ws + H->off_problems);
     const int32_t* unit_prefix = reinterpret_cast<const int32_t*>(ws + H->off_unit_prefix);
@@ -772,9 +515,21 @@ k_gemv_units_fine(const DeviceTables* __restrict__ tab, unsigned char* __restric
     }
 }
 
-// grouped_run must know a plan's mode without reading device memory: grouped_plan notes it here.
-static std::mutex g_plan_mu;
-static std::unordered_map<const void*, bool> g_plan_is_fine;
+// The persistent kernel of a planned list.  The plan in the workspace says which of the two modes it
+// was cut for (PlanHeader::off_fine), so a workspace can be copied or moved and still runs correctly:
+// the host needs no record of it.
+__global__ void __launch_bounds__(kUnitThreads, 1)
+k_gemv_units(const DeviceTables* __restrict__ tab, unsigned char* __restrict__ ws) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    pdl_release();
+    unsigned char* smem = stage_fast_tables(tab, smem_raw);
+    const uint32_t sm_tab = smem_u32(smem);
+    __syncthreads();  // the only CTA-wide barrier: tables are staged
+    pdl_wait();       // the plan's activation records (and zeroed counters) come from k_prepare_x
+    if (reinterpret_cast<const PlanHeader*>(ws)->off_fine) units_fine(ws, smem, sm_tab);
+    else units_coarse(ws, smem, sm_tab);
+}
+
 
 cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, size_t ws_bytes, cudaStream_t s) {
     if (ws_bytes < grouped_workspace_bytes(problems_host, count)) return cudaErrorInvalidValue;
@@ -868,10 +623,6 @@ cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, 
     // pageable source: the runtime stages it before returning, so the buffer can be freed
     if (e == cudaSuccess) e = cudaMemcpyAsync(ws_dev, buf, meta, cudaMemcpyHostToDevice, s);
     free(buf);
-    if (e == cudaSuccess) {
-        std::lock_guard<std::mutex> lock(g_plan_mu);
-        g_plan_is_fine[ws_dev] = fine_mode;
-    }
     return e;
 }
 
@@ -903,30 +654,14 @@ cudaError_t grouped_run(void* ws_dev, const void* table, cudaStream_t s) {
     int sms = 0;
     cudaError_t e = device_sms(&sms);
     if (e != cudaSuccess) return e;
-    static bool attr_set[64] = {false};
-    int dev = 0;
-    cudaGetDevice(&dev);
     const uint32_t smem = kTableSmemBytes + kUnitWarps * kRedFloats * 4 + kUnitWarps * 3072;
-    if (!attr_set[dev]) {
-        e = cudaFuncSetAttribute(k_gemv_units, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(k_gemv_units_fine, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-        if (e != cudaSuccess) return e;
-        attr_set[dev] = true;
-    }
-    bool fine_mode = false;
-    {
-        std::lock_guard<std::mutex> lock(g_plan_mu);
-        auto it = g_plan_is_fine.find(ws_dev);
-        if (it != g_plan_is_fine.end()) fine_mode = it->second;
-    }
+    static PerDeviceOnce once;
+    e = once.run([smem] { return cudaFuncSetAttribute(k_gemv_units, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)); });
+    if (e != cudaSuccess) return e;
     e = launch_pdl(k_prepare_x, sms * 2, 256, 0, s, static_cast<unsigned char*>(ws_dev));
     if (e != cudaSuccess) return e;
-    if (fine_mode)
-        return launch_pdl(k_gemv_units_fine, sms, kUnitThreads, smem, s, static_cast<const DeviceTables*>(table),
-                          static_cast<unsigned char*>(ws_dev));
     return launch_pdl(k_gemv_units, sms, kUnitThreads, smem, s, static_cast<const DeviceTables*>(table),
-                      static_cast<const unsigned char*>(ws_dev));
+                      static_cast<unsigned char*>(ws_dev));
 }
 
 }  // namespace tetra

@@ -28,8 +28,18 @@ cudaError_t launch_decode_packed(const void* packed, const void* table, int8_t* 
 cudaError_t launch_gemv_paper(const void* codes, size_t row_stride, const float* row_scales, const void* table,
                               const void* x, float* y, int N, int K, int batch, const void* tail, cudaStream_t s);
 
-// Fast GEMV of one matrix (x and y advanced per batch column inside); no scratch memory.
-cudaError_t launch_gemv_fast(const Problem& single, int batch, int max_blocks, const void* table, cudaStream_t s);
+// One matrix or a short list of matrices in a single launch, no scratch memory (the kernel behind
+// tetra_gemv, tetra_gemv_tail and tetra_gemv_list).  `batch` activation vectors per matrix, x and y
+// advanced by K and N per vector.
+constexpr int kListMax = 8;
+struct ListDesc {
+    int32_t count;
+    int32_t total_groups;               // eight-row groups of all matrices
+    int32_t group_prefix[kListMax + 1]; // row groups before matrix i
+    int32_t max_blocks;                 // largest number of words per row in the list
+    Problem problems[kListMax];
+};
+cudaError_t launch_gemv_list(const ListDesc& list, int batch, const void* table, cudaStream_t s);
 
 // Planned list of batch-1 products.  grouped_plan writes descriptors and prefix
 // arrays to the workspace (once per list); grouped_run enqueues the activation

@@ -43,6 +43,18 @@ int scratch_address(void** out) {
     return TETRA_OK;
 }
 
+// The plan of one product, passed to the device BY VALUE: kernel parameters are copied when the
+// launch is enqueued (and, under stream capture, when the node is created), so nothing points at
+// host memory that may be gone by the time the work runs.
+struct PlanBlob {
+    unsigned char bytes[256];
+};
+
+__global__ void k_write_plan(unsigned char* __restrict__ scratch, const PlanBlob blob) {
+    for (unsigned i = threadIdx.x; i < sizeof(PlanBlob) / 4; i += blockDim.x)
+        reinterpret_cast<uint32_t*>(scratch)[i] = reinterpret_cast<const uint32_t*>(blob.bytes)[i];
+}
+
 }  // namespace
 
 extern "C" int tetra_gemv_noalloc(const void* codes, const float* row_scales, const void* table, const void* x,
@@ -53,23 +65,26 @@ extern "C" int tetra_gemv_noalloc(const void* codes, const float* row_scales, co
     if (!aligned(codes, 16) || !aligned(table, 16) || !aligned(row_scales, 4) || !aligned(y, 4) || !aligned(x, 2) ||
         (tail && !aligned(tail, 2)))
         return TETRA_ERR_ALIGN;
+    // words per row, by the same rule as tetra_gemv_tail: a row must hold at least one word
+    const int B = (tail || K % 24 == 0) ? K / 24 : (K + 23) / 24;
+    if (B <= 0) return TETRA_ERR_SHAPE;
     const Problem problem{codes, row_scales, x, (K % 24) ? tail : nullptr, y, N, K};
-    if (single_plan_scratch_bytes((K + 23) / 24) > kNoAllocScratchBytes) return TETRA_ERR_SIZE;
+    if (single_plan_scratch_bytes(B) > kNoAllocScratchBytes) return TETRA_ERR_SIZE;
 
     void* scratch = nullptr;
     const int rc = scratch_address(&scratch);
     if (rc != TETRA_OK) return rc;
 
-    // The plan of this one product goes to the head of the array; the pre-pass
-    // kernel then rewrites the activation records behind it.  Nothing in the
-    // array has to start at zero: every byte the kernels read is written by this
-    // call first, whatever an earlier call left there.
-    unsigned char meta[256];
-    if (single_plan_meta_bytes() > sizeof meta) return TETRA_ERR_SIZE;
-    single_plan_fill(problem, meta);
+    // The plan of this one product goes to the head of the array (written by a one-block kernel from
+    // its own parameters); the pre-pass kernel then rewrites the activation records behind it.
+    // Nothing in the array has to start at zero: every byte the kernels read is written by this call
+    // first, whatever an earlier call left there.
+    PlanBlob blob;
+    static_assert(sizeof blob.bytes >= 256, "plan blob");
+    if (single_plan_meta_bytes() > sizeof blob.bytes) return TETRA_ERR_SIZE;
+    single_plan_fill(problem, blob.bytes);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // pageable source: the runtime has taken its copy of `meta` when the call returns
-    if (cudaMemcpyAsync(scratch, meta, single_plan_meta_bytes(), cudaMemcpyHostToDevice, s) != cudaSuccess)
-        return TETRA_ERR_CUDA;
+    k_write_plan<<<1, 64, 0, s>>>(static_cast<unsigned char*>(scratch), blob);
+    if (cudaGetLastError() != cudaSuccess) return TETRA_ERR_CUDA;
     return grouped_run(scratch, table, s) == cudaSuccess ? TETRA_OK : TETRA_ERR_CUDA;
 }

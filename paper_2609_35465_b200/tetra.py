@@ -17,6 +17,7 @@ BLOCK = 24
 WORD_BYTES = 6
 MAX_BATCH = 16
 PAPER_TABLE_BYTES = 18816
+LIST_MAX = 8
 
 
 class TetraError(RuntimeError):
@@ -54,6 +55,7 @@ def lib():
         L.tetra_decode_packed.argtypes = [vp, vp, vp, vp, i32, i32, vp]
         L.tetra_gemv.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp]
         L.tetra_gemv_tail.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, vp, vp]
+        L.tetra_gemv_list.argtypes = [vp, i32, vp, vp]
         L.tetra_grouped_workspace_bytes.argtypes = [vp, i32]
         L.tetra_grouped_workspace_bytes.restype = sz
         L.tetra_gemv_grouped_plan.argtypes = [vp, i32, vp, sz, vp]
@@ -171,6 +173,11 @@ def make_problems(items):
                          it["tail"].data_ptr() if it.get("tail") is not None else None,
                          it["y"].data_ptr(), it["N"], it["K"])
     return arr
+
+
+def tetra_gemv_list(problems, table, stream=None):
+    """Batch-1 products of a short list (ctypes array from make_problems, at most LIST_MAX) in one launch."""
+    _check(lib().tetra_gemv_list(problems, len(problems), _ptr(table), _stream(stream)), "tetra_gemv_list")
 
 
 def tetra_grouped_workspace_bytes(problems) -> int:

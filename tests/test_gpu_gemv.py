@@ -220,3 +220,113 @@ def test_hostio_mapped_results(tt, table, orc):
     for i, it in enumerate(dp.items):
         ref = oracle_product(orc, dp.host_inputs(i), dp.gain)
         assert_gemv_close(dp.y_mapped.numpy()[it["yoff"]:it["yoff"] + it["N"]], ref, it["name"])
+
+
+# ---------------------------------------------------------------------------
+# tetra_gemv_list: a short list in one launch, no plan and no scratch memory
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("shapes_list", [
+    [(1024, 4096, True), (256, 4096, True), (256, 4096, True)],                        # q, k, v of a layer, scaled down
+    [(520, 2560, True)],                                                               # one matrix, ragged rows
+    [(33, 24 * 31 + 5, False), (7, 48, True), (1, 24, True), (9, 24 * 33, True)],      # tiny: several matrices per CTA
+    [(40, 49152, True), (300, 24 * 64, True)],                                         # more columns than the image holds
+    [(300, 24 * 513, True), (264, 12288, True)],                                       # the sixteen-warp configuration
+    [(8 * i + 3, 24 * (i + 1) + i, i % 2 == 0) for i in range(8)],                     # the longest list, every rule
+])
+def test_gemv_list_matches_oracle(tt, table, orc, shapes_list):
+    mats = [make_matrix(39, 100 * i + N, N, K, tm) for i, (N, K, tm) in enumerate(shapes_list)]
+    devs = [upload(tt, table, m) for m in mats]
+    problems = tt.make_problems(devs)
+    tt.tetra_gemv_list(problems, table)
+    torch.cuda.synchronize()
+    first = [d["y"].cpu().numpy().copy() for d in devs]
+    for d in devs:
+        d["y"].fill_(float("nan"))
+    tt.tetra_gemv_list(problems, table)                    # the same bits on a second run
+    torch.cuda.synchronize()
+    for m, d, f in zip(mats, devs, first):
+        y = d["y"].cpu().numpy()[0]
+        assert np.array_equal(y, f[0])
+        ref = oracle_product(orc, m, GAIN)
+        assert_gemv_close(y, ref, "list %dx%d" % (m["N"], m["K"]))
+        assert np.max(np.abs(y - ref["y"]) / np.maximum(ref["abssum"], 1e-30)) < 1e-5
+
+
+def test_gemv_list_rejects_long_lists(tt, table):
+    m = make_matrix(39, 1, 8, 24, True)
+    devs = [upload(tt, table, m) for _ in range(tt.LIST_MAX + 1)]
+    problems = tt.make_problems(devs)
+    assert tt.lib().tetra_gemv_list(problems, len(problems), table.data_ptr(), None) == -2
+    assert tt.lib().tetra_gemv_list(problems, 0, table.data_ptr(), None) == -2
+
+
+# ---------------------------------------------------------------------------
+# a plan describes itself: the workspace can be moved
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("shapes_list", [
+    [(1024, 4096, True), (33, 749, False)],                                            # fine mode
+    [(40, 49152, True), (3000, 24 * 64, True), (16, 49152 - 24, True)],                # coarse mode
+])
+def test_planned_workspace_can_be_copied_to_another_address(tt, table, orc, shapes_list):
+    mats = [make_matrix(40, 100 * i + N, N, K, tm) for i, (N, K, tm) in enumerate(shapes_list)]
+    devs = [upload(tt, table, m) for m in mats]
+    problems = tt.make_problems(devs)
+    ws = torch.empty(tt.tetra_grouped_workspace_bytes(problems), dtype=torch.uint8, device="cuda")
+    tt.tetra_gemv_grouped_plan(problems, ws)
+    torch.cuda.synchronize()
+    moved = torch.empty(ws.numel() + 4096, dtype=torch.uint8, device="cuda")[2048:2048 + ws.numel()]
+    moved.copy_(ws)
+    ws.fill_(0xA5)                                         # the place where the plan was made is gone
+    del ws
+    tt.tetra_gemv_grouped_run(moved, table)
+    torch.cuda.synchronize()
+    for m, d in zip(mats, devs):
+        assert_gemv_close(d["y"].cpu().numpy()[0], oracle_product(orc, m, GAIN), "moved plan %dx%d" % (m["N"], m["K"]))
+
+
+# ---------------------------------------------------------------------------
+# non-finite activations
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("bad", [float("nan"), float("inf"), -float("inf")])
+def test_non_finite_activations_give_nan_rows_on_every_entry_point(tt, table, bad):
+    """A NaN or an infinity among the activations of a block column must not come out as a finite number:
+    every row reads every column, so every row is NaN (documented in the header)."""
+    N, K = 264, 24 * 40 + 16
+    m = make_matrix(41, 7, N, K, True, batch=3)
+    m["x"][1, 24 * 17 + 5] = np.float16(bad)               # vector 1 only
+    d = upload(tt, table, m)
+
+    def check(y, what):
+        assert np.isfinite(y[0]).all() and np.isfinite(y[2]).all(), what
+        assert np.isnan(y[1]).all(), what
+
+    check(run_fast(tt, table, m, d), "tetra_gemv_tail")
+    ws = torch.empty(tt.tetra_batched_workspace_bytes(N, K), dtype=torch.uint8, device="cuda")
+    yb = torch.zeros((3, N), dtype=torch.float32, device="cuda")
+    tt.tetra_gemv_batched(d["codes"], d["row_scales"], table, d["x"], yb, N, K, 3, d["tail"], ws)
+    torch.cuda.synchronize()
+    check(yb.cpu().numpy(), "tetra_gemv_batched")
+    # one vector at a time: list, planned list, no-allocation entry point
+    ys = {name: torch.zeros((3, N), dtype=torch.float32, device="cuda") for name in ("list", "grouped", "noalloc")}
+    for v in range(3):
+        item = dict(d, x=d["x"][v], y=ys["list"][v])
+        tt.tetra_gemv_list(tt.make_problems([item]), table)
+        item = dict(d, x=d["x"][v], y=ys["grouped"][v])
+        pr = tt.make_problems([item])
+        wsg = torch.empty(tt.tetra_grouped_workspace_bytes(pr), dtype=torch.uint8, device="cuda")
+        tt.tetra_gemv_grouped(pr, table, wsg)
+        tt.tetra_gemv_noalloc(d["codes"], d["row_scales"], table, d["x"][v], ys["noalloc"][v], N, K, d["tail"])
+        torch.cuda.synchronize()
+    for name, y in ys.items():
+        check(y.cpu().numpy(), name)
+
+
+def test_non_finite_tail_activation_follows_ieee(tt, table):
+    N, K = 64, 24 * 10 + 16
+    m = make_matrix(41, 8, N, K, True)
+    m["x"][0, 24 * 10 + 3] = np.float16("inf")             # multiplies tail weights only
+    d = upload(tt, table, m)
+    y = run_fast(tt, table, m, d)[0]
+    w = m["tail"][:, 3].astype(np.float32)
+    assert np.all(np.isinf(y[w != 0])) and np.all(np.sign(y[w != 0]) == np.sign(w[w != 0]))
+    assert np.all(np.isnan(y[w == 0]))

@@ -11,7 +11,7 @@ import pytest
 import torch
 
 from paper_2609_35465_b200 import synth
-from helpers import make_matrix
+from helpers import assert_gemv_close, make_matrix, oracle_product
 
 pytestmark = pytest.mark.gpu
 
@@ -23,7 +23,7 @@ def _device(tt, table, m):
                 tail=torch.from_numpy(m["tail"]).cuda() if m["tail"] is not None else None)
 
 
-def test_noalloc_matches_the_ordinary_entry_point_twice_in_a_row():
+def test_noalloc_matches_the_ordinary_entry_point_twice_in_a_row(orc):
     from paper_2609_35465_b200 import tetra as tt
     table = tt.tetra_build_table(synth.DEFAULT_GAIN)
     cases = [make_matrix(41, 1, 1024, 4096, True),      # 170 words per row + a tail of 16
@@ -40,6 +40,10 @@ def test_noalloc_matches_the_ordinary_entry_point_twice_in_a_row():
         # the two entry points sum in different orders: equal up to float32 rounding
         assert np.linalg.norm(a - b) <= 1e-5 * np.linalg.norm(a)
         assert np.max(np.abs(a - b)) <= 1e-4 * np.max(np.abs(a))
+        # and each against the FP64 oracle, within the tolerance of the GEMV tests
+        ref = oracle_product(orc, m, synth.DEFAULT_GAIN)
+        assert_gemv_close(b, ref, "noalloc %dx%d" % (m["N"], m["K"]))
+        assert_gemv_close(a, ref, "ordinary %dx%d" % (m["N"], m["K"]))
 
 
 def test_noalloc_rejects_sizes_beyond_its_fixed_scratch():
@@ -50,3 +54,8 @@ def test_noalloc_rejects_sizes_beyond_its_fixed_scratch():
                                      C.c_void_p(table.data_ptr()), C.c_void_p(buf.data_ptr()),
                                      C.c_void_p(buf.data_ptr()), 8, tt.NOALLOC_MAX_K + 24, None, None)
     assert rc == -6
+    # a tail pointer with K < 24 leaves no whole word in a row: rejected like tetra_gemv_tail does
+    rc = tt.lib().tetra_gemv_noalloc(C.c_void_p(buf.data_ptr()), C.c_void_p(buf.data_ptr()),
+                                     C.c_void_p(table.data_ptr()), C.c_void_p(buf.data_ptr()),
+                                     C.c_void_p(buf.data_ptr()), 8, 16, C.c_void_p(buf.data_ptr()), None)
+    assert rc == -2
