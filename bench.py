@@ -34,6 +34,16 @@ FALLBACK_HBM_GBS = 6650.0
 # for the 198.4 MB of the first 4 layers; every code byte is read once, so traffic grows in
 # proportion to the matrices read and the full pass is scaled by its byte count).
 TRAFFIC_PER_ALGORITHMIC_BYTE = 1.02
+# Warp-instructions of k_gemv_units per 32 blocks (one block per lane), by pipe, and wavefronts of the
+# shared-memory/L1 data pipe, from the same capture (smsp__inst_executed.sum and
+# sm__inst_executed_pipe_{alu,fmaheavy,lsu}.sum over the blocks processed / 32).
+KERNEL_COUNTERS = {"instr": 85.9, "alu": 40.1, "fmaheavy": 32.0, "lsu": 9.6, "wavefronts": 21.0}
+
+
+def issue_bound_gbs(sm_mhz, sms=148):
+    """Rate at which the kernel would consume code bytes if every issue slot were used: four schedulers
+    per SM, one warp-instruction per cycle each, KERNEL_COUNTERS['instr'] per 32 blocks of 6 bytes."""
+    return sms * 4 * sm_mhz * 1e6 / KERNEL_COUNTERS["instr"] * 32 * 6 / 1e9
 
 
 def measured_peak():
@@ -112,7 +122,7 @@ def timed(torch, fn, steps, warmup, stream):
 def oracle_sample(dp, orc, layers, threads, compare_with=None):
     """Times the CPU oracle on the first `layers` layers' matrices of the pass.
     Returns (seconds, bytes processed, worst ratio to the tolerance)."""
-    from tests.helpers import oracle_product  # the tolerance lives with the tests
+    from oracle.check import ABS_COEF, ABS_FLOOR, oracle_product
     per_layer = 7
     items = list(range(min(len(dp.items), layers * per_layer)))
     inputs = [dp.host_inputs(i) for i in items]
@@ -126,7 +136,7 @@ def oracle_sample(dp, orc, layers, threads, compare_with=None):
         for i, ref in zip(items, refs):
             it = dp.items[i]
             y = compare_with[it["yoff"]:it["yoff"] + it["N"]].astype(np.float64)
-            bound = 1e-3 * ref["termnorm"] + 1e-6
+            bound = ABS_COEF * ref["termnorm"] + ABS_FLOOR
             worst = max(worst, float(np.max(np.abs(y - ref["y"]) / bound)))
     return dt, nbytes, worst, len(items)
 
@@ -137,7 +147,7 @@ def run_reference(args, rank, world):
         return
     import oracle
     from paper_2609_35465_b200 import shapes, synth
-    from tests.helpers import make_matrix, oracle_product
+    from oracle.check import make_matrix, oracle_product
     orc = oracle.get()
     model = shapes.MODELS[args.model]
     mats = model.layer_matrices()               # one layer per step: a bounded sample of the pass
@@ -263,19 +273,30 @@ def main():
             torch.cuda.synchronize()
 
     # ---- headline: the whole pass as one persistent grouped launch ---------
+    # Rounds of exactly `steps` passes each, CUDA events around every round; as many rounds as it takes to
+    # time half a second of work (one round when `steps` alone covers that).  The reported step time is
+    # the median round's.
     for _ in range(args.warmup):
         dp.run_grouped()
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(args.steps):
-        dp.run_grouped()
-    e1.record(stream)
-    barrier()
+    round_ms = []
+    total_ms = 0.0
+    while True:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            dp.run_grouped()
+        e1.record(stream)
+        barrier()
+        t = ranks.max_over_ranks(e0.elapsed_time(e1), device="cuda")
+        round_ms.append(t / args.steps)
+        total_ms += t
+        if total_ms >= 500.0 or len(round_ms) >= 200:
+            break
     clocks = sampler.stop()
-    ms = ranks.max_over_ranks(e0.elapsed_time(e1) / args.steps, device="cuda")
+    ms = float(np.median(round_ms))
     y_grouped = dp.y_all.cpu().numpy().copy()
 
     # ---- end to end: activations from pinned host memory, results back to it
@@ -311,7 +332,10 @@ def main():
         "bits_per_weight_read": dp.algorithmic_bytes * 8 / sum(m.N * m.K for m in mats),
         "algorithmic_bytes_per_pass": dp.algorithmic_bytes,
         "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": 2 * args.steps * len(round_ms),
+        "timed_rounds": {"rounds": len(round_ms), "steps_per_round": args.steps, "timed_ms_total": total_ms,
+                         "ms_per_step_median": ms, "ms_per_step_best": float(min(round_ms)),
+                         "ms_per_step_worst": float(max(round_ms))},
         "clocks": clocks,
         "e2e": {"value": dp.algorithmic_bytes / (e2e_ms * 1e-3) / 1e9 * world, "unit": UNIT,
                 "ms_per_step": e2e_ms,
@@ -326,7 +350,14 @@ def main():
                      "frac": gbs / peak, "peak_kind": peak_kind + " copy bandwidth",
                      "traffic": (None if TRAFFIC_PER_ALGORITHMIC_BYTE is None
                                  else TRAFFIC_PER_ALGORITHMIC_BYTE * dp.algorithmic_bytes),
-                     "limiter": "ALU pipe (PRMT/LOP3/SHF, 64 lanes/clk/SM), not HBM: see DESIGN.md"},
+                     "limiter": "instruction issue, not HBM: %.1f warp-instructions per 32 blocks (logic/permute "
+                                "pipe %.1f, integer multiply-add pipe %.1f, load/store %.1f; both arithmetic pipes "
+                                "take one warp-instruction every two cycles per SM sub-partition); shared-memory "
+                                "data pipe %.0f wavefronts per 32 blocks" % (
+                                    KERNEL_COUNTERS["instr"], KERNEL_COUNTERS["alu"], KERNEL_COUNTERS["fmaheavy"],
+                                    KERNEL_COUNTERS["lsu"], KERNEL_COUNTERS["wavefronts"]),
+                     "issue_bound_gbs": issue_bound_gbs(clocks.get("sm_max_mhz") or 1965),
+                     "counters_per_32_blocks": KERNEL_COUNTERS},
         "paper_context": {"L40S_tokens_per_s": [113.8, 95.0, 57.2], "L40S_bits_per_weight": 2.148,
                           "L40S_kernel_GBps": 278},
     }
@@ -344,31 +375,49 @@ def main():
         assert np.linalg.norm(y_single - y_grouped) <= 1e-5 * np.linalg.norm(y_grouped), \
             "per-matrix launches differ from the planned run"
         arms["paper_design_stream_ms"] = timed(torch, dp.run_paper_design, max(3, reps // 5), 2, stream)
-        # the pass as a model would issue it: per layer four planned lists in stream order (q, k, v | o | gate, up |
-        # down: the matrices inside a list share their input and are independent, the lists depend on each
-        # other), every list planned once, the whole sequence replayed from one CUDA graph
+        # the pass as a model would issue it: per layer four dependency steps in stream order (q, k, v | o |
+        # gate, up | down: the matrices of a step share their input and are independent, the steps depend on
+        # each other), the whole sequence replayed from one CUDA graph.  Each step is one tetra_gemv_list
+        # launch; for comparison, the same steps as planned lists (two launches each).
         if not args.layers or args.layers >= 1:
+            steps_of_layer = ((0, 3), (3, 4), (4, 6), (6, 7))
+            lists = [tetra_mod.make_problems(dp.items[lo + a:lo + b])
+                     for lo in range(0, len(dp.items), 7) for a, b in steps_of_layer]
+
+            def run_lists(stream=None):
+                for pr in lists:
+                    tetra_mod.tetra_gemv_list(pr, dp.table, stream=stream)
+            dp.y_all.zero_()
+            run_lists()
+            torch.cuda.synchronize()
+            y_lists = dp.y_all.cpu().numpy()
+            assert np.linalg.norm(y_lists - y_grouped) <= 1e-5 * np.linalg.norm(y_grouped), \
+                "list launches differ from the planned run"
+            gl_ = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gl_, stream=torch.cuda.Stream()):
+                run_lists(stream=torch.cuda.current_stream())
+            arms["layer_sequence_graph_ms"] = timed(torch, gl_.replay, reps, 3, stream)
+            arms["layer_sequence_stream_ms"] = timed(torch, run_lists, reps, 3, stream)
+            del gl_
             seq = []
-            for lo in range(0, len(dp.items), 7):
-                for a, b in ((0, 3), (3, 4), (4, 6), (6, 7)):
-                    pr = tetra_mod.make_problems(dp.items[lo + a:lo + b])
-                    wsq = torch.empty(max(16, tetra_mod.tetra_grouped_workspace_bytes(pr)), dtype=torch.uint8, device="cuda")
-                    tetra_mod.tetra_gemv_grouped_plan(pr, wsq)
-                    seq.append((pr, wsq))
+            for pr in lists:
+                wsq = torch.empty(max(16, tetra_mod.tetra_grouped_workspace_bytes(pr)), dtype=torch.uint8, device="cuda")
+                tetra_mod.tetra_gemv_grouped_plan(pr, wsq)
+                seq.append(wsq)
             torch.cuda.synchronize()
 
             def run_sequence(stream=None):
-                for _, wsq in seq:
+                for wsq in seq:
                     tetra_mod.tetra_gemv_grouped_run(wsq, dp.table, stream=stream)
             run_sequence()
             gs_ = torch.cuda.CUDAGraph()
             with torch.cuda.graph(gs_, stream=torch.cuda.Stream()):
                 run_sequence(stream=torch.cuda.current_stream())
-            arms["layer_sequence_graph_ms"] = timed(torch, gs_.replay, reps, 3, stream)
-            arms["layer_sequence_stream_ms"] = timed(torch, run_sequence, reps, 3, stream)
-            out["layer_sequence"] = {"lists_per_pass": len(seq), "launches_per_pass": 2 * len(seq),
-                                     "note": "four dependent planned lists per layer (q,k,v | o | gate,up | down)"}
-            del gs_
+            arms["layer_sequence_planned_lists_graph_ms"] = timed(torch, gs_.replay, reps, 3, stream)
+            out["layer_sequence"] = {"steps_per_pass": len(lists), "launches_per_pass": len(lists),
+                                     "note": "four dependent steps per layer (q,k,v | o | gate,up | down), one "
+                                             "tetra_gemv_list launch each; planned lists take two launches each"}
+            del gs_, seq
             dp.run_grouped()
             torch.cuda.synchronize()
         # 20 rounds of ten planned passes each: median and best round (the paper reports the median of its rounds)
@@ -387,27 +436,70 @@ def main():
             if not k.startswith("no_weights"):
                 arms[k.replace("_ms", "_GBps")] = dp.algorithmic_bytes / (arms[k] * 1e-3) / 1e9
         out["other_arms"] = arms
+        for k in ("layer_sequence_graph_ms", "per_matrix_graph_ms", "no_weights_control_graph_ms"):
+            if k in arms:
+                out[k] = arms[k]       # beside `value`: the pass in model order, and one launch per matrix
         dp.run_grouped()
         torch.cuda.synchronize()
 
         # microseconds per matrix of the single-matrix entry point (tetra_gemv_tail), per shape of a layer:
-        # 12 distinct copies of the shape replayed from a CUDA graph, so no launch re-reads L2-resident codes
+        # distinct copies of the shape, together more than twice the 126 MB L2, replayed from a CUDA graph, so
+        # no launch reads L2-resident codes
         peak_now = measured_peak()[0]
-        per_matrix = {}
-        for m in model.layer_matrices():
-            one = DevicePass([shapes.Matrix("%s%d" % (m.name, i), m.N, m.K) for i in range(12)], seed=args.seed + 7)
+        L2_BYTES = 126e6
+
+        def copies_for(nbytes):
+            return int(max(12, min(400, np.ceil(2.2 * L2_BYTES / nbytes))))
+
+        def time_shape(mats_of_copy, run_name):
+            """mats_of_copy: shapes of one copy; returns (microseconds per copy, bytes per copy, copies)."""
+            probe = sum(m.N * (m.blocks * 6 + m.ntail * 2 + 8) + m.K * 2 for m in mats_of_copy)
+            copies = copies_for(probe)
+            one = DevicePass([shapes.Matrix("%s_%d" % (m.name, i), m.N, m.K) for i in range(copies) for m in mats_of_copy],
+                             seed=args.seed + 7)
+            n = len(mats_of_copy)
+            if run_name == "per_matrix":
+                fn = one.run_per_matrix
+            else:
+                groups = [tetra_mod.make_problems(one.items[i * n:(i + 1) * n]) for i in range(copies)]
+
+                def fn(stream=None):
+                    for pr in groups:
+                        tetra_mod.tetra_gemv_list(pr, one.table, stream=stream)
             for _ in range(2):
-                one.run_per_matrix()
+                fn()
             gg = torch.cuda.CUDAGraph()
             with torch.cuda.graph(gg, stream=torch.cuda.Stream()):
-                one.run_per_matrix(stream=torch.cuda.current_stream())
-            us = timed(torch, gg.replay, 20, 3, stream) * 1e3 / 12
-            b = one.items[0]["bytes"]
-            per_matrix[m.name] = {"N": m.N, "K": m.K, "us": us, "GBps": b / us / 1e3,
-                                  "weights_per_s": m.N * m.K / us * 1e6, "frac_of_measured_peak": b / us / 1e3 / peak_now,
-                                  "roofline_us": b / peak_now / 1e3}
+                fn(stream=torch.cuda.current_stream())
+            us = timed(torch, gg.replay, 20, 3, stream) * 1e3 / copies
+            b = sum(it["bytes"] for it in one.items[:n])
             del one, gg
+            torch.cuda.empty_cache()
+            return us, b, copies
+
+        def figure(mats_of_copy, run_name):
+            us, b, copies = time_shape(mats_of_copy, run_name)
+            return {"us": us, "GBps": b / us / 1e3, "algorithmic_bytes": b, "distinct_copies": copies,
+                    "weights_per_s": sum(m.N * m.K for m in mats_of_copy) / us * 1e6,
+                    "frac_of_measured_peak": b / us / 1e3 / peak_now, "roofline_us": b / peak_now / 1e3}
+
+        per_matrix = {}
+        for m in model.layer_matrices():
+            per_matrix[m.name] = dict(figure([m], "per_matrix"), N=m.N, K=m.K)
         out["per_matrix_tetra_gemv"] = per_matrix
+        # BASELINE configs 0 and 1: the single 2048 x 2304 matrix (one launch), and one Qwen3-4B-shaped layer
+        # (seven matrices) as its four dependency steps, one tetra_gemv_list launch each
+        l4 = shapes.QWEN3_4B.layer_matrices()
+        cfg1 = {"us_per_layer": 0.0, "algorithmic_bytes": 0, "launches": 4}
+        for a, b in ((0, 3), (3, 4), (4, 6), (6, 7)):
+            f = figure(l4[a:b], "list")
+            cfg1["us_per_layer"] += f["us"]
+            cfg1["algorithmic_bytes"] += f["algorithmic_bytes"]
+            cfg1["+".join(m.name for m in l4[a:b])] = {"us": f["us"], "GBps": f["GBps"]}
+        cfg1["GBps"] = cfg1["algorithmic_bytes"] / cfg1["us_per_layer"] / 1e3
+        cfg1["frac_of_measured_peak"] = cfg1["GBps"] / peak_now
+        out["configs"] = {"config0_2048x2304": dict(figure([shapes.CONFIG0], "per_matrix"), N=shapes.CONFIG0.N, K=shapes.CONFIG0.K),
+                          "config1_qwen3_4b_layer": cfg1}
 
         # batch sweep on the down_proj shape (N 4096, K 12288): tetra_gemv_batched (decode once, tensor-core
         # contraction) against one tetra_gemv_tail launch per vector; 12 distinct code copies per CUDA graph
@@ -514,8 +606,24 @@ def main():
                 continue
             mm = shapes.MODELS[name]
             od = DevicePass(mm.all_matrices(), seed=args.seed + 11)
+            # correctness first (Sec. 5.1): sampled rows of every matrix of the pass against the oracle
+            od.run_grouped()
+            torch.cuda.synchronize()
+            y_od = od.y_all.cpu().numpy()
+            import oracle
+            from oracle.check import gemv_errors, oracle_product
+            worst_od = 0.0
+            for i, it in enumerate(od.items):
+                rows = np.unique(np.concatenate([[0, it["N"] - 1],
+                                                 np.random.default_rng(args.seed + i).integers(0, it["N"], 6)]))
+                ref = oracle_product(oracle.get(), od.host_inputs(i, rows), od.gain)
+                rel, worst = gemv_errors(y_od[it["yoff"] + rows], ref)
+                worst_od = max(worst_od, worst, rel / 1e-3)
+            if worst_od > 1.0:
+                raise SystemExit("%s pass outside the tolerance on sampled rows: %.3f" % (name, worst_od))
             t = timed(torch, od.run_grouped, 30, 3, stream)
             others[name] = {"matrices": len(od.items), "algorithmic_bytes": od.algorithmic_bytes, "ms_per_pass": t,
+                            "sampled_rows_worst_fraction_of_tolerance": worst_od,
                             "GBps": od.algorithmic_bytes / (t * 1e-3) / 1e9,
                             "frac_of_measured_peak": od.algorithmic_bytes / (t * 1e-3) / 1e9 / peak_now,
                             "weights_per_s": sum(x.N * x.K for x in mm.all_matrices()) / (t * 1e-3)}

@@ -52,14 +52,21 @@ def test_qwen3_8b_full_pass_sampled_rows(orc):
     assert np.array_equal(dp.y_host.numpy()[used], y[used])
 
 
-def test_qwen3_14b_layers_sampled_rows(orc):
-    """Config 3 shapes (hidden 5120, intermediate 17408: 213 and 725 words per row, tails of 8)."""
+def test_qwen3_14b_full_pass_sampled_rows(orc):
+    """Config 3: all 280 matrices of the Qwen3-14B-shaped pass (hidden 5120, intermediate 17408: 213 and
+    725 words per row, tails of 8; 3.35 GB) in one planned run, sampled rows of every matrix."""
     from paper_2609_35465_b200.workload import DevicePass
-    mats = shapes.QWEN3_14B.all_matrices()[:14]
-    dp = DevicePass(mats, seed=3)
+    dp = DevicePass(shapes.QWEN3_14B.all_matrices(), seed=3)
+    assert len(dp.items) == 280
+    dp.y_all.fill_(float("nan"))
     dp.run_grouped()
     torch.cuda.synchronize()
-    _check_sampled(dp, orc, range(len(mats)), rows_per_matrix=4, seed=3)
+    y = dp.y_all.cpu().numpy()
+    used = np.zeros(len(y), dtype=bool)
+    for it in dp.items:
+        used[it["yoff"]:it["yoff"] + it["N"]] = True
+    assert np.isfinite(y[used]).all()                     # every output row was written
+    _check_sampled(dp, orc, range(len(dp.items)), rows_per_matrix=4, seed=3)
 
 
 def test_qwen3_4b_layer_zero_pad_rule(orc):
@@ -94,3 +101,31 @@ def test_down_proj_batch_sweep_sampled_rows(orc, batch):
         mm = dict(N=len(rows), K=m.K, B=m.blocks, ntail=0, codes=host_codes, sigma=sigma[rows], x=x, tail=None)
         ref = oracle_product(orc, mm, synth.DEFAULT_GAIN, batch_index=b, threads=1)
         assert_gemv_close(yh[b][rows], ref, "batch %d column %d" % (batch, b))
+
+
+@pytest.mark.parametrize("batch", shapes.CONFIG4_BATCHES)
+def test_down_proj_batched_sampled_rows(orc, batch):
+    """Config 4 through tetra_gemv_batched (decode once, tensor-core contraction): the shape and the batch
+    sizes the benchmark's sweep times.  Rows: first and last, the rows around the 16- and 32-row tile edges,
+    around the boundaries of the 16-warp tile groups (512 rows) and around the CTA ranges' cuts, and random
+    ones; every vector of the batch."""
+    from paper_2609_35465_b200 import tetra as tt
+    m = shapes.CONFIG4
+    table = tt.tetra_build_table(synth.DEFAULT_GAIN)
+    codes = synth.codes_torch(6, 2, m.N, m.blocks, device="cuda")
+    packed = tt.tetra_pack_codes(codes, table, m.N, m.blocks)
+    sigma = synth.row_scales(6, 2, m.N)
+    x = synth.activations(6, 2, m.K, batch)
+    y = torch.full((batch, m.N), float("nan"), dtype=torch.float32, device="cuda")
+    tt.tetra_gemv_batched(packed, torch.from_numpy(sigma).cuda(), table, torch.from_numpy(x).cuda(), y, m.N, m.K,
+                          batch, None)
+    torch.cuda.synchronize()
+    yh = y.cpu().numpy()
+    assert np.isfinite(yh).all()
+    edges = [0, 1, 15, 16, 31, 32, 33, 511, 512, 513, 1023, 1024, 2047, 2048, 3071, 3072, 3583, 3584, 4094, 4095]
+    rows = np.unique(np.concatenate([edges, np.random.default_rng(batch).integers(0, m.N, 12)]))
+    host_codes = np.stack([synth.words_to_bytes(synth.words(6, 2, m.blocks, int(r) * m.blocks)) for r in rows])
+    for b in range(batch):
+        mm = dict(N=len(rows), K=m.K, B=m.blocks, ntail=0, codes=host_codes, sigma=sigma[rows], x=x, tail=None)
+        ref = oracle_product(orc, mm, synth.DEFAULT_GAIN, batch_index=b, threads=4)
+        assert_gemv_close(yh[b][rows], ref, "batched, batch %d vector %d" % (batch, b))
