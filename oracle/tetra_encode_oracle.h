@@ -27,7 +27,14 @@
  * decode -> encode round trips (cosine 1); never worse than sampled codewords;
  * the retention of Sec. 3.5 on Gaussian blocks lies between the paper's
  * figure for its non-exhaustive search and the figure of the 24-dimensional
- * ball; the gain rule against a direct evaluation of the error.
+ * ball; the gain rule against a direct evaluation of the error.  Two pins that
+ * do not share this search's decomposition, both through to_decode_word only:
+ * planted optima (codebook points from deep rows -- ranks 2 to 4, the class-1
+ * half of the middle list, both parities -- turned by 3 degrees, where any two
+ * codebook directions are at least 15.9 degrees apart, must come back as the
+ * planted direction), and a brute-force neighbourhood (none of the ~10,000
+ * words that differ from the answer in one field has a larger cosine; over a
+ * million words in all).
  */
 #ifndef TETRA_ENCODE_ORACLE_H
 #define TETRA_ENCODE_ORACLE_H

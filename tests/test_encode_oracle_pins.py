@@ -104,3 +104,44 @@ def test_retention_on_gaussian_blocks(orc):
     D = ((w - what) ** 2).mean()
     retention = 0.5 * np.log2(1.0 / D) / 2.0 * 100.0
     assert 88.80 <= retention <= 91.98, retention
+
+
+# ---------------------------------------------------------------------------
+# Pins that do not share the search's decomposition (per-section tables joined over the trellis): both go
+# through the word decoder only.
+# ---------------------------------------------------------------------------
+def test_planted_optima_deep_in_the_lists(orc):
+    """Codebook points from deep rows (ranks 2-4, the class-1 half of the middle list, the last entries of the
+    lists, both parities), turned by 3 degrees: any two codebook directions are at least 15.9 degrees apart,
+    so the search must come back with the planted direction."""
+    from encode_cases import deep_words, direction_cosines, planted_blocks
+    words = deep_words(orc, 2000, seed=5)
+    rows = np.asarray(orc.rows, dtype=np.uint32)
+    assert ((words >> np.uint64(11)) & np.uint64(2047) >= np.uint64(orc.n0)).sum() >= 900
+    w, Y = planted_blocks(orc, words, seed=6)
+    found, cos = encode.encode_blocks(w)
+    assert np.all(np.abs(cos - np.cos(np.deg2rad(3.0))) <= 1e-9)          # the value of the optimum
+    c, Y2 = direction_cosines(orc, found & MASK48, Y)                     # direction of the word it returns
+    assert np.all(c >= 1 - 1e-12)
+    ranks = np.stack([(rows >> np.uint32(4 * j)) & np.uint32(15) for j in range(8)], axis=1).max(axis=1)
+    i1 = (words & np.uint64(2047)).astype(np.int64) + 2048 * ((words >> np.uint64(46)) & np.uint64(1)).astype(np.int64)
+    assert {2, 3, 4} <= set(ranks[i1].tolist())                           # the planted rows do reach ranks 2, 3, 4
+
+
+def test_no_single_field_neighbour_beats_the_search(orc):
+    """Brute force through the word decoder around the search's answer: every word that differs from it in one
+    field (all 2048 values of each row index, all 4096 trellis paths, the other parity/class pairs), about
+    10,000 words per block, over a million in all; none may have a larger cosine."""
+    from encode_cases import direction_cosines, single_field_neighbours
+    n = 104
+    w = synth.normal(12, 3, 20, n * 24).reshape(n, 24).astype(np.float64)
+    w[0, 8:] = 0
+    w[1] = np.abs(w[1])
+    found, cos = encode.encode_blocks(w)
+    total = 0
+    for k in range(n):
+        nb = single_field_neighbours(found[k])
+        c, _ = direction_cosines(orc, nb, w[k])
+        assert c.max() <= cos[k] + 1e-12, (k, c.max(), cos[k])
+        total += len(nb)
+    assert total >= 1_000_000

@@ -111,3 +111,30 @@ def test_encode_retention_at_full_size(orc):
     assert abs(got.min() - golden["min_cosine"]) <= 1e-5
     assert abs(retention - golden["retention_percent"]) <= 2e-3
     assert 88.80 <= retention <= 91.98
+
+
+def test_gpu_planted_optima_deep_in_the_lists(orc):
+    """The planted-optimum pin of the oracle, on the GPU search: points from deep rows turned by 3 degrees come
+    back as words of exactly the planted direction."""
+    from encode_cases import deep_words, direction_cosines, planted_blocks
+    words = deep_words(orc, 4000, seed=7)
+    w, Y = planted_blocks(orc, words, seed=8)
+    found, cos = _encode_gpu(w)
+    c, _ = direction_cosines(orc, found & MASK47, Y)
+    assert np.all(c >= 1 - 1e-12)
+    assert np.max(np.abs(cos - np.cos(np.deg2rad(3.0)))) <= 1e-5
+
+
+def test_gpu_no_single_field_neighbour_beats_the_search(orc):
+    from encode_cases import direction_cosines, single_field_neighbours
+    n = 104
+    w = synth.normal(12, 4, 20, n * 24).reshape(n, 24).astype(np.float32)
+    found, cos = _encode_gpu(w)
+    got, _, _ = _fp64_cosine(orc, found, w.astype(np.float64))
+    total = 0
+    for k in range(n):
+        nb = single_field_neighbours(found[k])
+        c, _ = direction_cosines(orc, nb, w[k].astype(np.float64))
+        assert c.max() <= got[k] * (1 + 1e-5), (k, c.max(), got[k])   # float32 correlations: near-ties may swap
+        total += len(nb)
+    assert total >= 1_000_000
