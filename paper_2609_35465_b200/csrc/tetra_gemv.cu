@@ -409,7 +409,7 @@ __device__ __forceinline__ void units_coarse(const unsigned char* __restrict__ w
 // Each unit leaves eight partial row sums in the scratch area and bumps its row group's counter; the
 // unit that finds all the other slices done adds them up in slice order (fixed order, no waiting,
 // no floating-point atomics), applies the row scale and the tail, and stores.
-__device__ __forceinline__ void units_fine(unsigned char* __restrict__ ws, unsigned char* smem, uint32_t sm_tab) {
+__device__ __noinline__ void units_fine(unsigned char* __restrict__ ws, unsigned char* smem, uint32_t sm_tab) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float* red = reinterpret_cast<float*>(smem + kFastBytes) + warp * kRedFloats;
     const PlanHeader* H = reinterpret_cast<const PlanHeader*>(ws);
