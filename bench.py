@@ -189,6 +189,9 @@ def main():
     ap.add_argument("--encode-only", type=int, default=0, metavar="BLOCKS",
                     help="profiling runs: two tetra_encode_blocks launches on this many Gaussian blocks, nothing else, "
                          "no JSON line")
+    ap.add_argument("--list-only", type=int, default=0, metavar="LAYERS",
+                    help="profiling runs: the dependency steps of this many layers (q,k,v | o | gate,up | down), one "
+                         "tetra_gemv_list launch each, three rounds, nothing else, no JSON line")
     ap.add_argument("--q4-only", default="", metavar="N,K,G,BATCH",
                     help="profiling runs: three tetra_q4_gemv launches on one synthetic matrix, nothing else, "
                          "no JSON line")
@@ -242,6 +245,16 @@ def main():
         yq = torch.empty((qB, qN), dtype=torch.float32, device="cuda")
         for _ in range(3):
             tetra.tetra_q4_gemv(pk, xq, yq, qN, qK, qG, qB)
+        torch.cuda.synchronize()
+        return
+    if args.list_only:
+        from paper_2609_35465_b200 import tetra
+        lp = DevicePass(shapes.MODELS[args.model].all_matrices()[:7 * args.list_only], seed=args.seed + 5)
+        lists = [tetra.make_problems(lp.items[lo + a:lo + b]) for lo in range(0, len(lp.items), 7)
+                 for a, b in ((0, 3), (3, 4), (4, 6), (6, 7))]
+        for _ in range(3):
+            for pr in lists:
+                tetra.tetra_gemv_list(pr, lp.table)
         torch.cuda.synchronize()
         return
     if args.batched_only:
