@@ -192,6 +192,9 @@ def main():
     ap.add_argument("--list-only", type=int, default=0, metavar="LAYERS",
                     help="profiling runs: the dependency steps of this many layers (q,k,v | o | gate,up | down), one "
                          "tetra_gemv_list launch each, three rounds, nothing else, no JSON line")
+    ap.add_argument("--q4-list-only", type=int, default=0, metavar="LAYERS",
+                    help="profiling runs: three tetra_q4_list_run passes over the v, o and down shapes of this many "
+                         "layers (groups of 128), nothing else, no JSON line")
     ap.add_argument("--q4-only", default="", metavar="N,K,G,BATCH",
                     help="profiling runs: three tetra_q4_gemv launches on one synthetic matrix, nothing else, "
                          "no JSON line")
@@ -231,6 +234,24 @@ def main():
         enc_table = tetra.tetra_build_table(synth.DEFAULT_GAIN)
         for _ in range(2):
             tetra.tetra_encode_blocks(wd, enc_table)
+        torch.cuda.synchronize()
+        return
+    if args.q4_list_only:
+        from paper_2609_35465_b200 import synth, tetra
+        mdl = shapes.MODELS[args.model]
+        kv_dim, q_dim = mdl.kv_heads * mdl.head_dim, mdl.q_heads * mdl.head_dim
+        qitems = []
+        for layer in range(args.q4_list_only):
+            for qN, qK in ((kv_dim, mdl.hidden), (mdl.hidden, q_dim), (mdl.hidden, mdl.intermediate)):
+                qn = torch.from_numpy(synth.q4_nibbles(args.seed + 17, qN, min(qN, 4096), qK)).cuda()
+                sc, of = synth.q4_scales_offsets(args.seed + 17, qN, qN, qK // 128)
+                qitems.append(dict(packed=tetra.tetra_q4_pack(qn, torch.from_numpy(sc).cuda(), torch.from_numpy(of).cuda(),
+                                                              qN, qK, 128), N=qN, K=qK,
+                                   x=torch.from_numpy(synth.activations(args.seed + 17, layer, qK, 1)[0]).cuda(),
+                                   y=torch.empty(qN, dtype=torch.float32, device="cuda")))
+        qws = tetra.tetra_q4_list_plan(tetra.make_q4_problems(qitems), 128)
+        for _ in range(3):
+            tetra.tetra_q4_list_run(qws, 128)
         torch.cuda.synchronize()
         return
     if args.q4_only:
@@ -590,6 +611,42 @@ def main():
                         "bits_per_weight": 8.0 * packs[0].numel() / (qN * qK)}
             del packs, gg, qn, sc, of
             torch.cuda.empty_cache()
+        # the same projection shapes as ONE planned list (v, o and down of every layer: 3 x layers matrices,
+        # distinct copies, more than L2 together), three launches per pass (tetra_q4_list_run)
+        qitems = []
+        for layer in range(model.layers):
+            for name, qN, qK, qG, _ in q4_shapes[:3]:
+                rows_src = min(qN, 4096)
+                qn = torch.from_numpy(synth.q4_nibbles(args.seed + 17, qN, rows_src, qK)).cuda()
+                sc, of = synth.q4_scales_offsets(args.seed + 17, qN, qN, qK // qG)
+                pk = tetra.tetra_q4_pack(qn, torch.from_numpy(sc).cuda(), torch.from_numpy(of).cuda(), qN, qK, qG)
+                qitems.append(dict(packed=pk, N=qN, K=qK,
+                                   x=torch.from_numpy(synth.activations(args.seed + 17, layer, qK, 1)[0]).cuda(),
+                                   y=torch.empty(qN, dtype=torch.float32, device="cuda")))
+                del qn
+        qprob = tetra.make_q4_problems(qitems)
+        qws = tetra.tetra_q4_list_plan(qprob, 128)
+        torch.cuda.synchronize()
+        t_end = time.time() + 0.5
+        while time.time() < t_end:
+            tetra.tetra_q4_list_run(qws, 128)
+            torch.cuda.synchronize()
+        ms_list = timed(torch, lambda: tetra.tetra_q4_list_run(qws, 128), 20, 3, stream)
+        # spot check against the single-matrix entry point (itself checked against the oracle in the tests)
+        it0 = qitems[5]
+        y1 = torch.empty((1, it0["N"]), dtype=torch.float32, device="cuda")
+        tetra.tetra_q4_gemv(it0["packed"], it0["x"].reshape(1, -1), y1, it0["N"], it0["K"], 128, 1)
+        torch.cuda.synchronize()
+        assert torch.linalg.norm(y1[0] - it0["y"]) <= 1e-5 * torch.linalg.norm(y1[0]), "q4 list differs from q4 gemv"
+        nbytes_list = sum(it["packed"].numel() + 2 * it["K"] + 4 * it["N"] for it in qitems)
+        q4["planned_list_v_o_down"] = {"matrices": len(qitems), "algorithmic_bytes": nbytes_list, "ms_per_pass": ms_list,
+                                       "GBps": nbytes_list / (ms_list * 1e-3) / 1e9,
+                                       "frac_of_measured_peak": nbytes_list / (ms_list * 1e-3) / 1e9 / peak_now,
+                                       "single_launches_sum_ms": sum(q4[n]["us"] for n in ("v_proj", "o_proj", "down_proj"))
+                                                                 * model.layers * 1e-3,
+                                       "launches_per_pass": 3}
+        del qitems, qws
+        torch.cuda.empty_cache()
         out["q4_gemv"] = q4
 
         # encoder search on Gaussian blocks (Sec. 3.5): exact largest-cosine point per block on the GPU, and the

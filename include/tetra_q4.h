@@ -66,6 +66,37 @@ int tetra_q4_gemv(const void *packed_dev, const void *x_dev, float *y_dev, int N
 int tetra_q4_rows(const void *packed_dev, const int32_t *ids_dev, int count, void *out_dev, int N, int K, int G,
                   void *stream);
 
+/* One product of a list call: packed_dev as written by tetra_q4_pack, x_dev float16 [K] (16-byte
+ * aligned), y_dev float32 [N]. */
+typedef struct {
+    const void *packed;
+    const void *x;
+    float *y;
+    int32_t N;
+    int32_t K;
+} tetra_q4_problem;
+
+#define TETRA_Q4_LIST_MAX 4096
+
+/* Batch-1 products of a list of independent 4-bit matrices with one group size G (the int4
+ * projections of a token pass, Sec. 4.1, 4.3) from one persistent grid: the chunks of all matrices
+ * form one stream that the warps cut into equal contiguous ranges, so nothing is paid per matrix.
+ * The list is planned once and run many times:
+ *   tetra_q4_list_workspace_bytes  size of the scratch buffer (descriptors, per-group sums of the
+ *                                  activations, partial strips); 0 for a rejected list;
+ *   tetra_q4_list_plan             writes the descriptors (problems_host is read before the call
+ *                                  returns; call it outside stream capture);
+ *   tetra_q4_list_run              one step, three launches: group sums of every x, the stream, the
+ *                                  sum of the strips that two warps share (in warp order).
+ * workspace_dev: 256-byte aligned device memory owned by the caller; it belongs to the plan until the
+ * last run using it has completed, runs that share it must not overlap on the GPU, and it may be
+ * copied to other device memory (the plan describes itself) on the device it was planned for.
+ * Same result definition, arithmetic and tolerance as tetra_q4_gemv; bit-identical from run to run. */
+size_t tetra_q4_list_workspace_bytes(const tetra_q4_problem *problems_host, int count, int G);
+int tetra_q4_list_plan(const tetra_q4_problem *problems_host, int count, int G, void *workspace_dev,
+                       size_t workspace_bytes, void *stream);
+int tetra_q4_list_run(void *workspace_dev, int G, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

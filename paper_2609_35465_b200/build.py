@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtetra_b200.so")
-SOURCES = ["tetra_tables.cpp", "tetra_decode.cu", "tetra_gemv.cu", "tetra_list.cu", "tetra_batched.cu", "tetra_api.cu", "tetra_noalloc.cu", "q4_gemv.cu", "tetra_encode.cu"]
+SOURCES = ["tetra_tables.cpp", "tetra_decode.cu", "tetra_gemv.cu", "tetra_list.cu", "tetra_batched.cu", "tetra_api.cu", "tetra_noalloc.cu", "q4_gemv.cu", "q4_list.cu", "tetra_encode.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--use_fast_math"]

@@ -24,6 +24,11 @@ class TetraError(RuntimeError):
     pass
 
 
+class Q4Problem(C.Structure):
+    """Mirror of tetra_q4_problem."""
+    _fields_ = [("packed", C.c_void_p), ("x", C.c_void_p), ("y", C.c_void_p), ("N", C.c_int32), ("K", C.c_int32)]
+
+
 class Problem(C.Structure):
     """Mirror of tetra_problem."""
     _fields_ = [("codes", C.c_void_p), ("row_scales", C.c_void_p), ("x", C.c_void_p),
@@ -74,6 +79,10 @@ def lib():
         L.tetra_q4_pack.argtypes = [vp, vp, vp, vp, sz, i32, i32, i32, vp]
         L.tetra_q4_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
         L.tetra_q4_rows.argtypes = [vp, vp, i32, vp, i32, i32, i32, vp]
+        L.tetra_q4_list_workspace_bytes.argtypes = [vp, i32, i32]
+        L.tetra_q4_list_workspace_bytes.restype = sz
+        L.tetra_q4_list_plan.argtypes = [vp, i32, i32, vp, sz, vp]
+        L.tetra_q4_list_run.argtypes = [vp, i32, vp]
         _lib = L
     return _lib
 
@@ -290,3 +299,27 @@ def tetra_encode_blocks(w, table, sigma=None, want_cosine=True, stream=None):
     _check(lib().tetra_encode_blocks(_ptr(w), _ptr(sigma), _ptr(table), _ptr(codes), _ptr(cos), n, _stream(stream)),
            "tetra_encode_blocks")
     return codes, cos
+
+
+def make_q4_problems(items):
+    """items: iterable of dicts(packed, x, y, N, K) of device tensors -> ctypes array of tetra_q4_problem."""
+    items = list(items)
+    arr = (Q4Problem * len(items))()
+    for i, it in enumerate(items):
+        arr[i] = Q4Problem(it["packed"].data_ptr(), it["x"].data_ptr(), it["y"].data_ptr(), it["N"], it["K"])
+    return arr
+
+
+def tetra_q4_list_plan(problems, G: int, stream=None) -> torch.Tensor:
+    """Plans a list of 4-bit products (one group size); returns the workspace tensor to pass to the run."""
+    n = lib().tetra_q4_list_workspace_bytes(problems, len(problems), G)
+    if n == 0:
+        raise TetraError("tetra_q4_list_workspace_bytes: list rejected")
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+    _check(lib().tetra_q4_list_plan(problems, len(problems), G, _ptr(ws), ws.numel(), _stream(stream)),
+           "tetra_q4_list_plan")
+    return ws
+
+
+def tetra_q4_list_run(workspace: torch.Tensor, G: int, stream=None):
+    _check(lib().tetra_q4_list_run(_ptr(workspace), G, _stream(stream)), "tetra_q4_list_run")

@@ -56,6 +56,9 @@ def test_host_side_argument_checks(L):
     assert L.tetra_build_table(p16, 16, None, None) == -6                          # blob too small
     assert L.tetra_table_export(p16, 10) == -6
     assert L.tetra_gemv_grouped(None, 1, p16, p16, 48, None) == -1
+    assert L.tetra_gemv_list(None, 1, p16, None) == -1                               # no descriptors
+    assert L.tetra_gemv_list(p16, 1, None, None) == -1                               # no table
+    assert L.tetra_gemv_list(p16, 9, p16, None) in (-1, -2)                          # zeroed descriptors / too long
     assert L.tetra_gemv_grouped_run(None, p16, None) == -1
     assert L.tetra_codes_bytes(4096, 170) == 4096 * 170 * 6
     assert L.tetra_codes_bytes(9, 3) == 2 * 48 * 3                                  # rows pad to 8

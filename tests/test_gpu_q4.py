@@ -149,3 +149,67 @@ def test_q4_head_full_size_sampled_rows():
         d = got[:, rows] - want
         assert np.linalg.norm(d) / np.linalg.norm(want) <= REL_L2
         assert np.max(np.abs(d) / (ABS_COEF * tn + ABS_FLOOR)) <= 1.0
+
+
+# ---------------------------------------------------------------------------
+# tetra_q4_list_*: a list of matrices from one persistent grid
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("G,shapes_list", [
+    (128, [(1024, 4096), (4096, 4096), (4096, 12288)]),                 # v, o, down of a Qwen3-8B-shaped layer
+    (128, [(37, 1152), (16, 128), (300, 2560), (1, 256), (64, 1024)]),  # ragged rows, tiny matrices
+    (64, [(129, 2560), (2048, 5120)]),                                  # groups of 64
+    (128, [(32, 65536)]),                                               # one strip cut across hundreds of warps
+    (64, [(40, 65536), (33, 64)]),
+])
+def test_q4_list_matches_oracle(G, shapes_list):
+    import torch
+    from oracle import q4 as oq
+    from paper_2609_35465_b200 import tetra
+    mats, items = [], []
+    for i, (N, K) in enumerate(shapes_list):
+        q, s, o, packed = _device_matrix(24, 100 * i + N + K, N, K, G)
+        x = synth.activations(24, i, K, 1)
+        y = torch.full((N,), float("nan"), dtype=torch.float32, device="cuda")
+        mats.append((q, s, o, x, N, K))
+        items.append(dict(packed=packed, x=torch.from_numpy(x[0]).cuda(), y=y, N=N, K=K))
+    problems = tetra.make_q4_problems(items)
+    ws = tetra.tetra_q4_list_plan(problems, G)
+    tetra.tetra_q4_list_run(ws, G)
+    torch.cuda.synchronize()
+    first = [it["y"].cpu().numpy().copy() for it in items]
+    for it in items:
+        it["y"].fill_(float("nan"))
+    moved = torch.empty(ws.numel() + 1024, dtype=torch.uint8, device="cuda")[512:512 + ws.numel()]
+    moved.copy_(ws)                                          # the plan describes itself: run it from a copy
+    ws.fill_(0x5A)
+    tetra.tetra_q4_list_run(moved, G)
+    torch.cuda.synchronize()
+    for (q, s, o, x, N, K), it, f in zip(mats, items, first):
+        got = it["y"].cpu().numpy()
+        assert np.array_equal(got, f)                        # bit-identical from run to run
+        want, tn = oq.gemv(q, s, o, x, N, K, G, 1)
+        assert np.isfinite(got).all()
+        rel = np.linalg.norm(got - want[0]) / max(np.linalg.norm(want[0]), 1e-300)
+        assert rel <= REL_L2, rel
+        assert np.max(np.abs(got - want[0]) / (ABS_COEF * tn[0] + ABS_FLOOR)) <= 1.0
+        # and the single-matrix entry point gives the same values up to float32 summation order
+        y1 = torch.empty((1, N), dtype=torch.float32, device="cuda")
+        tetra.tetra_q4_gemv(it["packed"], it["x"].reshape(1, -1), y1, N, K, G, 1)
+        torch.cuda.synchronize()
+        assert np.linalg.norm(y1.cpu().numpy()[0] - got) <= 1e-5 * max(np.linalg.norm(got), 1e-30)
+
+
+def test_q4_list_rejects_bad_lists():
+    import torch
+    from paper_2609_35465_b200 import tetra
+    q, s, o, packed = _device_matrix(25, 1, 64, 256, 128)
+    x = torch.zeros(256, dtype=torch.float16, device="cuda")
+    y = torch.zeros(64, dtype=torch.float32, device="cuda")
+    ok = tetra.make_q4_problems([dict(packed=packed, x=x, y=y, N=64, K=256)])
+    assert tetra.lib().tetra_q4_list_workspace_bytes(ok, 1, 128) > 0
+    assert tetra.lib().tetra_q4_list_workspace_bytes(ok, 1, 96) == 0          # group size
+    assert tetra.lib().tetra_q4_list_workspace_bytes(ok, 0, 128) == 0         # empty list
+    bad = tetra.make_q4_problems([dict(packed=packed, x=x, y=y, N=64, K=192)])
+    assert tetra.lib().tetra_q4_list_workspace_bytes(bad, 1, 128) == 0        # K not a multiple of G
+    ws = torch.empty(16, dtype=torch.uint8, device="cuda")
+    assert tetra.lib().tetra_q4_list_plan(ok, 1, 128, ws.data_ptr(), 16, None) == -6
