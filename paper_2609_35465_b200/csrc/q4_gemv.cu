@@ -23,6 +23,7 @@
 #include "../../include/tetra_q4.h"
 #include "q4_common.cuh"
 #include "tetra_device.cuh"
+#include "tetra_launch.h"
 
 namespace tetra {
 namespace {
@@ -352,17 +353,11 @@ cudaError_t launch_q4_variant(const void* packed, const void* x, float* y, int N
     int grid = strips < kQ4CtasPerSm * sms ? strips : kQ4CtasPerSm * sms;
     const size_t smem = size_t(groups) * 64 + size_t(kQ4Warps) * 2048 + size_t(kQ4Warps) * DEPTH * q4_chunk_bytes(G) +
                         (XS ? size_t(batch) * (size_t(K) * 2 + 16) : 0);
-    static bool attr_set[64] = {false};  // per instantiation and device
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    static PerDeviceOnce once;  // per instantiation
+    cudaError_t e = once.run([] {
+        return cudaFuncSetAttribute(k_q4_gemv<G, DEPTH, XS>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kQ4SmemLimit));
+    });
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!attr_set[dev]) {
-        e = cudaFuncSetAttribute(k_q4_gemv<G, DEPTH, XS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 int(kQ4SmemLimit));
-        if (e != cudaSuccess) return e;
-        attr_set[dev] = true;
-    }
     if (smem > kQ4SmemLimit) return cudaErrorInvalidValue;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

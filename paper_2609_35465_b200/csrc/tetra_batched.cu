@@ -387,22 +387,19 @@ static cudaError_t launch_variant(const void* codes, const float* row_scales, co
 
 cudaError_t launch_gemv_batched(const void* codes, const float* row_scales, const void* table, const void* x,
                                 float* y, int N, int K, int batch, const void* tail, void* ws, cudaStream_t s) {
-    static bool attr_set[64] = {false};
-    int dev = 0, sms = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int sms = 0;
+    cudaError_t e = device_sms(&sms);
     if (e != cudaSuccess) return e;
     if (sms > 1024) sms = 1024;
     const uint32_t smem = kTableSmemBytes + kBatWarps * kBatWarpSmem + 2 * kPassTiles * 2 * kBatColBytesPerGroup;
-    if (!attr_set[dev]) {
-        e = cudaFuncSetAttribute(k_gemv_batched<1, TETRA_BAT_RB1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(k_gemv_batched<2, TETRA_BAT_RB2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-        if (e != cudaSuccess) return e;
-        attr_set[dev] = true;
-    }
+    static PerDeviceOnce once;
+    e = once.run([smem] {
+        cudaError_t r = cudaFuncSetAttribute(k_gemv_batched<1, TETRA_BAT_RB1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (r == cudaSuccess)
+            r = cudaFuncSetAttribute(k_gemv_batched<2, TETRA_BAT_RB2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        return r;
+    });
+    if (e != cudaSuccess) return e;
     const int B = tail ? K / 24 : (K + 23) / 24;
     const __half* xh = static_cast<const __half*>(x);
     const __half* tl = static_cast<const __half*>(tail);

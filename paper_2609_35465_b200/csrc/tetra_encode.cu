@@ -491,19 +491,13 @@ k_encode(const float* __restrict__ w, const float* __restrict__ sigma, const Dev
 
 cudaError_t launch_encode(const float* w, const float* sigma, const void* table, unsigned char* codes, float* cosine,
                           size_t nblocks, cudaStream_t s) {
-    static bool attr_set[64] = {false};
-    int dev = 0, sms = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int sms = 0;
+    cudaError_t e = device_sms(&sms);
     if (e != cudaSuccess) return e;
     const int smem = int(sizeof(EncShared));
-    if (!attr_set[dev]) {
-        e = cudaFuncSetAttribute(k_encode, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        attr_set[dev] = true;
-    }
+    static PerDeviceOnce once;
+    e = once.run([smem] { return cudaFuncSetAttribute(k_encode, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); });
+    if (e != cudaSuccess) return e;
     const unsigned grid = unsigned(nblocks < size_t(sms) ? nblocks : size_t(sms));
     k_encode<<<grid, kEncThreads, smem, s>>>(w, sigma, static_cast<const DeviceTables*>(table), codes, cosine, nblocks);
     return cudaGetLastError();

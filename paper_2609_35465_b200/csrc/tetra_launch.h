@@ -4,7 +4,38 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 namespace tetra {
+
+// One-time set-up per device (function attributes and the like), safe when several host threads
+// make their first call at once.
+class PerDeviceOnce {
+public:
+    template <typename F>
+    cudaError_t run(F&& setup) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(mu_);
+        if (!done_[dev]) {
+            e = setup();
+            if (e != cudaSuccess) return e;
+            done_[dev] = true;
+        }
+        return cudaSuccess;
+    }
+
+private:
+    static constexpr int kMaxDevices = 64;
+    std::mutex mu_;
+    bool done_[kMaxDevices] = {};
+};
+
+
+// Multiprocessors of the current device (cached per device, thread-safe).
+cudaError_t device_sms(int* sms);
 
 // Device-side view of one product; same layout as tetra_problem in tetra.h.
 struct Problem {
