@@ -6,20 +6,23 @@
 // cores (mma.sync m16n8k32); everything around it (field extraction, table
 // lookups, per-block scale, FP32 accumulation) is the batch-1 decoder.
 //
-// Thread layout: a warp owns RB row blocks of 16 rows, a CTA of 16 warps a group of 16 such row tiles,
-// and the CTA walks the block columns 8 / RB at a time; such a (tile group, column group) cell is the
-// unit of work, and the CTAs take equal contiguous ranges of the tile-group-major cell order.  In one
-// pass lane l decodes four blocks (row l % 16 of row block j % RB, column l / 16 + 2 (j / RB), j = 0..3),
-// writes each block's 24 int8 coordinates as a row of a shared-memory tile (coordinates 24..31 are zero)
-// and the block's scale next to it; the warp then loads the tiles as MMA A fragments with ldmatrix and
-// multiplies them with the three int8 planes of the activations' 24-bit fixed-point image (B fragments,
-// read once per column and used for the warp's RB row blocks).  The image of a pass's columns is built
-// by the CTA itself, in shared memory, during the pass before.  The int32 results of the planes are
+// Thread layout: a warp owns two row blocks of 16 rows, a CTA of 16 warps a tile group of 512 rows, and a
+// warp walks the block columns four at a time; such a (tile group, four columns) cell is the unit of work,
+// and the CTAs take equal contiguous ranges of the tile-group-major cell order.  The codes of a warp's pass
+// (four row groups x three parts x four columns) arrive through the warp's own cp.async ring, one pass
+// ahead.  In one pass lane l decodes four blocks (row l % 16 of row block j % 2, column l / 16 + 2 (j / 2),
+// j = 0..3) and writes each block's 24 int8 coordinates and its scale as a row of a shared-memory tile;
+// the warp then loads the tiles as MMA A fragments with ldmatrix and multiplies them with the three int8
+// planes of the activations' 24-bit fixed-point image (B fragments, read once per column and used for both
+// row blocks; coordinates 24..31 of the image are zero, so the tile's bytes there do not matter).  The image
+// of the CTA's next 32 (column, vector group) pairs is built by the CTA itself, in shared memory: once for
+// most calls (behind the first pass's decode), again behind two CTA barriers when the CTA's range is
+// longer; between those the warps never wait for one another.  The int32 results of the planes are
 // combined exactly, converted once, scaled by block scale x activation step and added into FP32
 // accumulators that the lane keeps for its (row, vector) pairs: no cross-lane reduction is needed.  When a
 // CTA's range leaves a tile group, its partial sums go to the scratch area as one piece; a second, small
 // kernel adds the pieces of every tile group in CTA order (fixed order, no atomics, no flags), applies the
-// row scale and the tail.  The only waits are CTA barriers and griddepcontrol.wait.
+// row scale and the tail.  The only waits are CTA barriers, cp.async groups and griddepcontrol.wait.
 #include <cuda_fp16.h>
 
 #include "tetra_device.cuh"
@@ -44,8 +47,7 @@ constexpr int kPassTiles = 8;  // 16-row x 1-column tiles per warp and pass (fou
 // where the lane multiplies with vector 8 n + lane / 4, t = lane % 4, register h = 0 holds coordinates
 // 4 t .. 4 t + 3 and h = 1 coordinates 16 + 4 t .. 16 + 4 t + 3 (24..31 and unused vectors are zero), and
 // the steps are those of the lane's two result columns.  A column takes ng x 1 KiB (ng = 1 or 2 groups).
-// The image lives in shared memory only: the CTA builds the columns of its next pass while it works on the
-// current one.
+// The image lives in shared memory only: the CTA builds it for a chunk of its passes at a time.
 constexpr int kBatGroupWords = 2 * 32 * 4;
 
 // One thread per (block column of a pass, vector, t) builds the words of lane (vector % 8) * 4 + t: the
@@ -116,25 +118,16 @@ __device__ __forceinline__ void mma_s8u8(int (&d)[4], const uint32_t (&a)[4], ui
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(0));
 }
 
-// Words of the block (row, col) from the packed layout; rows at or beyond rows_padded are the origin.
-__device__ __forceinline__ void load_block_words(const unsigned char* __restrict__ codes, uint32_t col_end, int row,
-                                                 int rows_padded, uint32_t col, uint32_t B, uint32_t* w0,
-                                                 uint32_t* w1) {
-    if (row >= rows_padded || col >= col_end) {
-        *w0 = 0;
-        *w1 = 0;
-        return;
-    }
-    const uint32_t G = uint32_t(row) >> 3, r = uint32_t(row) & 7u;
-    const unsigned char* rec = codes + (size_t(G) * 3 * B + col) * 16;
-    *w0 = __ldg(reinterpret_cast<const uint32_t*>(rec + size_t(r >> 2) * B * 16 + (r & 3u) * 4));
-    *w1 = __ldg(reinterpret_cast<const unsigned short*>(rec + size_t(2) * B * 16 + r * 2));
-}
-
-constexpr int kTileRow = 48;                // bytes per tile row: 24 coordinates, 8 zeros, 16 pad
+constexpr int kTileRow = 48;                // bytes per tile row: 24 coordinates, scale, 20 pad
 constexpr int kTileBytes = 16 * kTileRow;   // (48-byte rows keep ldmatrix and the tile stores conflict-free)
-constexpr int kBatWarpSmem = kPassTiles * kTileBytes + kPassTiles * 64;  // coordinate tiles + block scales
-constexpr int kBatColBytesPerGroup = kBatGroupWords * 4;                 // image of one column, per ng
+constexpr int kBatWarpTiles = kPassTiles * kTileBytes;  // coordinate tiles (a row: 24 coordinates, the block scale, pad)
+constexpr int kBatColBytesPerGroup = kBatGroupWords * 4;                   // image of one column, per ng
+// Code ring of a warp: two slots of one pass (the warp's four row groups x three parts x four columns x 16
+// bytes); a row group takes 224 bytes, so that the loads of a pass (two row groups x two parts x two
+// columns x four words per instruction) fall into different banks.
+constexpr uint32_t kBatRingGroup = 224, kBatRingSlot = 4 * kBatRingGroup;
+constexpr int kBatWarpSmem = kBatWarpTiles + 2 * int(kBatRingSlot);
+constexpr int kImageGroups = 32;  // (column, vector group) pairs of the activation image held at a time: 32 KiB
 
 __device__ __forceinline__ void lds128(uint32_t saddr, uint32_t (&v)[4]) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(saddr));
@@ -145,63 +138,88 @@ __device__ __forceinline__ uint32_t cta_of_cell(uint32_t x, uint32_t ctas, uint3
     return uint32_t(((uint64_t(x) + 1) * ctas - 1) / cells);
 }
 
-// NG: vector groups of eight, 1 (batch <= 8) or 2.  RB: 16-row blocks per warp.
+// NG: vector groups of eight, 1 (batch <= 8) or 2.  A warp owns two 16-row blocks (RB = 2), the CTA's 16
+// warps a tile group of 512 rows; a cell is a tile group x four block columns, one pass of every warp.
+// The CTAs take equal contiguous ranges of the tile-group-major cell order.  Between the image barriers the
+// warps run on their own: codes arrive through the warp's cp.async ring one pass ahead.
 template <int NG, int RB>
 __global__ void __launch_bounds__(kBatThreads, 1)
 k_gemv_batched(const DeviceTables* __restrict__ tab, const unsigned char* __restrict__ codes,
                const __half* __restrict__ x, int N, int K, int B, int batch, float* __restrict__ partials, int tile_groups, int col_groups) {
-    constexpr int PC = kPassTiles / RB;  // block columns per pass
-    constexpr int kSlotBytes = PC * NG * kBatColBytesPerGroup;
+    static_assert(RB == 2, "the ring and the lane mapping are laid out for two row blocks per warp");
+    constexpr int PC = kPassTiles / RB;          // block columns per pass
+    constexpr int CP = kImageGroups / (PC * NG); // passes per image chunk
     constexpr int kPieceFloats = RB * 128 * NG;  // partial results of one warp: 16 RB rows x 8 NG vectors
     extern __shared__ __align__(16) unsigned char smem_raw[];
     pdl_release();
-    unsigned char* smem = stage_fast_tables(tab, smem_raw);
+    // the tables start towards shared memory first; they are waited for together with the first pass's codes
+    unsigned char* smem = stage_fast_tables_async(tab, smem_raw);
     const uint32_t sm_tab = smem_u32(smem);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // per warp: eight 16-row tiles of coordinates (tile rb * PC + column), then 8 x 16 block scales; after
-    // the warps' areas, two slots for the activation image of a column group
+    // per warp: eight 16-row tiles of coordinates and block scales (tile rb * PC + column), the code ring;
+    // after the warps' areas, the activation image of a chunk of passes
     unsigned char* tiles = smem + kFastBytes + warp * kBatWarpSmem;
-    float* scales = reinterpret_cast<float*>(tiles + kPassTiles * kTileBytes);
-    const uint32_t slots = smem_u32(smem + kFastBytes + kBatWarps * kBatWarpSmem);
+    const uint32_t ring = smem_u32(tiles) + uint32_t(kBatWarpTiles);
+    const uint32_t image = smem_u32(smem + kFastBytes + kBatWarps * kBatWarpSmem);
     const int row16 = lane & 15, colsel = lane >> 4;
-#pragma unroll
-    for (int j = 0; j < 4; ++j)  // coordinates 24..31 of every tile row stay zero for the whole kernel
-        *reinterpret_cast<uint2*>(tiles + (colsel + 2 * j) * kTileBytes + row16 * kTileRow + 24) = make_uint2(0u, 0u);
 
-    const int rows_padded = ((N + 7) / 8) * 8;
+    const int row_groups = (N + 7) / 8;
     const uint32_t Bu = uint32_t(B);
     const int g = lane >> 2, t4 = lane & 3;  // MMA fragment coordinates
     const uint32_t tile_addr = smem_u32(tiles);
     // ldmatrix: lane provides the address of row (lane % 8) of 8x8 matrix (lane / 8):
     // matrices = (rows 0-7, bytes 0-15), (rows 8-15, bytes 0-15), (rows 0-7, bytes 16-31), (rows 8-15, bytes 16-31)
     const uint32_t ldm_off = uint32_t((((lane >> 3) & 1) * 8 + (lane & 7)) * kTileRow + (lane >> 4) * 16);
+    // block j of the lane in a pass: row row16 of row block j % 2, column colsel + 2 (j / 2); its words in a slot
+    const uint32_t lane_w0 = uint32_t(row16 >> 3) * kBatRingGroup + uint32_t((row16 >> 2) & 1) * 64u + uint32_t(colsel) * 16u +
+                             uint32_t(row16 & 3) * 4u;
+    const uint32_t lane_w1 = uint32_t(row16 >> 3) * kBatRingGroup + 128u + uint32_t(colsel) * 16u + uint32_t(row16 & 7) * 2u;
+    // the lane's copies of a pass: 48 pieces of 16 bytes, (row group, part) = piece / 4, column = piece % 4
+    const uint32_t cp0_gp = uint32_t(lane >> 2), cp1_gp = 8u + uint32_t(lane >> 2), cp_col = uint32_t(lane & 3);
+    const uint32_t cp0_dst = (cp0_gp / 3u) * kBatRingGroup + (cp0_gp % 3u) * 64u + cp_col * 16u;
+    const uint32_t cp1_dst = (cp1_gp / 3u) * kBatRingGroup + (cp1_gp % 3u) * 64u + cp_col * 16u;
 
     const uint32_t ctas = gridDim.x, cells = uint32_t(tile_groups) * uint32_t(col_groups), CG = uint32_t(col_groups);
     const uint32_t cell_begin = uint32_t(uint64_t(blockIdx.x) * cells / ctas);
     const uint32_t cell_end = uint32_t((uint64_t(blockIdx.x) + 1) * cells / ctas);
     uint32_t tg = cell_begin / CG, cg = cell_begin - tg * CG;
 
-    // block j of the lane: row block j % RB, column colsel + 2 (j / RB) of the pass
-    auto load_pass = [&](uint32_t group_tg, uint32_t group_cg, uint32_t (&w0)[4], uint32_t (&w1)[4]) {
-        const int row0 = (int(group_tg) * kBatWarps + warp) * (16 * RB) + row16;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            load_block_words(codes, Bu, row0 + 16 * (j % RB), rows_padded, group_cg * PC + colsel + 2 * (j / RB), Bu,
-                             &w0[j], &w1[j]);
+    // the codes of the warp's pass in cell (ftg, fcg) into ring slot `slot`; what lies outside the matrix is zero
+    auto fetch = [&](uint32_t ftg, uint32_t fcg, uint32_t slot) {
+        const uint32_t G0 = (ftg * kBatWarps + uint32_t(warp)) * (2 * RB);  // first of the warp's four row groups
+        const uint32_t col = fcg * PC + cp_col;
+        const bool in = col < Bu;
+        const uint4* base = reinterpret_cast<const uint4*>(codes) + size_t(G0) * 3 * Bu + (in ? col : 0u);
+        const uint32_t dst = ring + slot * kBatRingSlot;
+        const bool have0 = in && G0 + cp0_gp / 3u < uint32_t(row_groups);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(dst + cp0_dst),
+                     "l"(have0 ? base + size_t(cp0_gp) * Bu : reinterpret_cast<const uint4*>(codes)), "r"(have0 ? 16u : 0u));
+        if (lane < 16) {
+            const bool have1 = in && G0 + cp1_gp / 3u < uint32_t(row_groups);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(dst + cp1_dst),
+                         "l"(have1 ? base + size_t(cp1_gp) * Bu : reinterpret_cast<const uint4*>(codes)), "r"(have1 ? 16u : 0u));
+        }
+        asm volatile("cp.async.commit_group;");
     };
-    uint32_t w0[4], w1[4];
-    if (cell_begin < cell_end) load_pass(tg, cg, w0, w1);
-    __syncthreads();
+    if (cell_begin < cell_end) fetch(tg, cg, 0);
+    else asm volatile("cp.async.commit_group;");
     pdl_wait();  // x may come from the preceding kernel; the partial results of an earlier call have been read
-    // image tasks: warp w < PC * NG builds the group (column w / NG of the pass, vectors 8 (w % NG) + lane / 4)
-    const bool image_warp = warp < PC * NG;
-    const int image_col = warp / NG, image_vec = 8 * (warp % NG) + (lane >> 2);
-    const uint32_t image_group = uint32_t(warp) * 1024u;
-    ImageTask task;
-    if (image_warp && cell_begin < cell_end) {
-        image_load(x, K, batch, int(cg) * PC + image_col, image_vec, lane & 3, task);
-        image_store(task, slots + image_group, image_vec, lane & 3);
-    }
+
+    // Image tasks of a chunk of CP passes: task (pass i of the chunk, column cs, vector group n) = a warp's worth
+    // of threads; the 16 warps take two tasks each.
+    auto image_task_load = [&](uint32_t first_cell, int id, ImageTask& T) {
+        const uint32_t cell = first_cell + uint32_t(id / (PC * NG));
+        if (cell < cell_end) image_load(x, K, batch, int(cell % CG) * PC + (id / NG) % PC, 8 * (id % NG) + (lane >> 2), lane & 3, T);
+    };
+    auto image_task_store = [&](uint32_t first_cell, int id, const ImageTask& T) {
+        const uint32_t cell = first_cell + uint32_t(id / (PC * NG));
+        if (cell < cell_end) image_store(T, image + uint32_t(id) * 1024u, 8 * (id % NG) + (lane >> 2), lane & 3);
+    };
+    ImageTask task0, task1;
+    image_task_load(cell_begin, warp, task0);
+    image_task_load(cell_begin, warp + kBatWarps, task1);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();  // tables staged, tile padding written
 
     float acc[RB][NG][4];
 #pragma unroll
@@ -212,37 +230,50 @@ k_gemv_batched(const DeviceTables* __restrict__ tab, const unsigned char* __rest
             for (int i = 0; i < 4; ++i) acc[rb][n][i] = 0.f;
 
     for (uint32_t cell = cell_begin; cell < cell_end; ++cell) {
-        const uint32_t slot = (cell - cell_begin) & 1u;
-        const int row_base = (int(tg) * kBatWarps + warp) * (16 * RB);
-        const bool active = row_base < N;  // warp-uniform
-        uint32_t cw0[4], cw1[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { cw0[j] = w0[j]; cw1[j] = w1[j]; }
+        const uint32_t pass = cell - cell_begin, slot = pass & 1u, in_chunk = pass % CP;
+        const bool active = (int(tg) * kBatWarps + warp) * (16 * RB) < N;  // warp-uniform
         uint32_t ntg = tg, ncg = cg + 1;
         if (ncg == CG) { ncg = 0; ++ntg; }
-        __syncthreads();  // this cell's image is complete; everyone has left the slot the next one goes to
-        const bool more = cell + 1 < cell_end;
-        if (more) {
-            if (image_warp) image_load(x, K, batch, int(ncg) * PC + image_col, image_vec, lane & 3, task);
-            load_pass(ntg, ncg, w0, w1);
+        if (in_chunk == 0 && pass > 0) {  // CTA-uniform: the image of the next chunk of passes replaces the old one
+            __syncthreads();
+            image_task_load(cell, warp, task0);
+            image_task_load(cell, warp + kBatWarps, task1);
+            image_task_store(cell, warp, task0);
+            image_task_store(cell, warp + kBatWarps, task1);
+            __syncthreads();
         }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncwarp();  // every lane's copies have landed, and every lane has left the other slot
+        if (cell + 1 < cell_end) fetch(ntg, ncg, slot ^ 1u);
         if (active) {
+            const uint32_t src = ring + slot * kBatRingSlot;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
+                uint32_t w0, w1;
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w0) : "r"(src + lane_w0 + (j % RB) * 2 * kBatRingGroup + (j / RB) * 32));
+                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(w1) : "r"(src + lane_w1 + (j % RB) * 2 * kBatRingGroup + (j / RB) * 32));
                 FastBlock fb;
-                fast_decode<false>(sm_tab, cw0[j], cw1[j], fb);
-                int n2 = 0;
+                fast_decode<false>(sm_tab, w0, w1, fb);
+                int n2 = int(fb.goff);  // the squared norm on top of the gain's column of the scale table: the scale's address
 #pragma unroll
                 for (int k = 0; k < 6; ++k) n2 = dp4a_ss(fb.y[k], fb.y[k], n2);
-                const float scale = lds32f(fb.goff | (uint32_t(n2) & 0x1F0u));  // gain[g] / sqrt(16 m)
+                const float scale = lds32f(uint32_t(n2));  // -gain[g] / sqrt(16 m), with -y in the tile
                 const int tile_id = (j % RB) * PC + 2 * (j / RB);  // + colsel
                 unsigned char* dst = tiles + (tile_id + colsel) * kTileBytes + row16 * kTileRow;
+                // coordinates 24..31 of a tile row meet zeros in the activation image, so those eight bytes
+                // need not be zero: the block's scale rides there
                 *reinterpret_cast<uint4*>(dst) = make_uint4(fb.y[0], fb.y[1], fb.y[2], fb.y[3]);
-                *reinterpret_cast<uint2*>(dst + 16) = make_uint2(fb.y[4], fb.y[5]);
-                scales[(tile_id + colsel) * 16 + row16] = scale;
+                *reinterpret_cast<uint4*>(dst + 16) = make_uint4(fb.y[4], fb.y[5], __float_as_uint(scale), 0u);
             }
+        }
+        if (pass == 0) {  // the first chunk's image: its loads were issued before the first pass was decoded
+            image_task_store(cell_begin, warp, task0);
+            image_task_store(cell_begin, warp + kBatWarps, task1);
+            __syncthreads();
+        }
+        if (active) {
             __syncwarp();
-            const uint32_t img = slots + slot * kSlotBytes + lane * 16;
+            const uint32_t img = image + in_chunk * (PC * NG * 1024u) + lane * 16;
 #pragma unroll
             for (int cs = 0; cs < PC; ++cs) {
                 uint32_t q0[NG][4], q1[NG][4];
@@ -258,7 +289,8 @@ k_gemv_batched(const DeviceTables* __restrict__ tab, const unsigned char* __rest
                     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                                  : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
                                  : "r"(tile_addr + tile_id * kTileBytes + ldm_off));
-                    const float s_lo = scales[tile_id * 16 + g], s_hi = scales[tile_id * 16 + g + 8];
+                    const float s_lo = *reinterpret_cast<const float*>(tiles + tile_id * kTileBytes + g * kTileRow + 24);
+                    const float s_hi = *reinterpret_cast<const float*>(tiles + tile_id * kTileBytes + (g + 8) * kTileRow + 24);
 #pragma unroll
                     for (int n = 0; n < NG; ++n) {
                         int dh[4], dm[4], dl[4];
@@ -295,7 +327,6 @@ k_gemv_batched(const DeviceTables* __restrict__ tab, const unsigned char* __rest
                         acc[rb][n][i + 1] = 0.f;
                     }
         }
-        if (more && image_warp) image_store(task, slots + (slot ^ 1u) * kSlotBytes + image_group, image_vec, lane & 3);
         tg = ntg;
         cg = ncg;
     }
@@ -309,20 +340,24 @@ k_combine_batched(const float* __restrict__ partials, const float* __restrict__ 
                   int B, int batch, int tile_groups, int col_groups, int ctas) {
     constexpr int kPieceFloats = RB * 128 * NG, kGroupRows = kBatWarps * 16 * RB;
     pdl_release();
-    pdl_wait();  // the pieces come from k_gemv_batched
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     const int v = idx % (8 * NG), r = idx / (8 * NG);
-    if (r >= N || v >= batch) return;
-    const uint32_t tg = uint32_t(r / kGroupRows), CG = uint32_t(col_groups);
-    const int warp = (r % kGroupRows) / (16 * RB), rt = r % (16 * RB);
+    const bool mine = r < N && v < batch;
+    // what does not depend on the pieces comes before the wait for k_gemv_batched
+    const int rr = mine ? r : 0;
+    const uint32_t tg = uint32_t(rr / kGroupRows), CG = uint32_t(col_groups);
+    const int warp = (rr % kGroupRows) / (16 * RB), rt = rr % (16 * RB);
     const uint32_t cells = uint32_t(tile_groups) * CG;
     const uint32_t first = cta_of_cell(tg * CG, uint32_t(ctas), cells);
     const uint32_t pieces = cta_of_cell(tg * CG + CG - 1, uint32_t(ctas), cells) - first + 1;
+    const float scale = mine ? __ldg(row_scales + r) : 0.f;
+    pdl_wait();  // the pieces come from k_gemv_batched
+    if (!mine) return;
     const float* p = partials + (size_t(first + tg) * kBatWarps + warp) * kPieceFloats + rt * (8 * NG) + v;
     float total = 0.f;
 #pragma unroll 8
     for (uint32_t k = 0; k < pieces; ++k) total += __ldcg(p + size_t(k) * kBatWarps * kPieceFloats);
-    float res = __ldg(row_scales + r) * total;
+    float res = scale * total;
     const int ntail = tail ? K % 24 : 0;
     for (int k = 0; k < ntail; ++k)
         res = fmaf(__half2float(tail[size_t(r) * ntail + k]), __half2float(x[size_t(v) * K + 24 * B + k]), res);
@@ -391,7 +426,7 @@ cudaError_t launch_gemv_batched(const void* codes, const float* row_scales, cons
     cudaError_t e = device_sms(&sms);
     if (e != cudaSuccess) return e;
     if (sms > 1024) sms = 1024;
-    const uint32_t smem = kTableSmemBytes + kBatWarps * kBatWarpSmem + 2 * kPassTiles * 2 * kBatColBytesPerGroup;
+    const uint32_t smem = kTableSmemBytes + kBatWarps * kBatWarpSmem + kImageGroups * kBatColBytesPerGroup;
     static PerDeviceOnce once;
     e = once.run([smem] {
         cudaError_t r = cudaFuncSetAttribute(k_gemv_batched<1, TETRA_BAT_RB1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
