@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_2609_35465_b200 import shapes, synth
-from helpers import assert_gemv_close, oracle_product
+from helpers import assert_gemv_close, make_matrix, oracle_product
 
 pytestmark = pytest.mark.gpu
 
@@ -129,3 +129,27 @@ def test_down_proj_batched_sampled_rows(orc, batch):
         mm = dict(N=len(rows), K=m.K, B=m.blocks, ntail=0, codes=host_codes, sigma=sigma[rows], x=x, tail=None)
         ref = oracle_product(orc, mm, synth.DEFAULT_GAIN, batch_index=b, threads=4)
         assert_gemv_close(yh[b][rows], ref, "batched, batch %d vector %d" % (batch, b))
+
+
+@pytest.mark.parametrize("batch", [5, 16])
+def test_batched_long_cta_ranges_sampled_rows(orc, batch):
+    """8192 x 9232 through tetra_gemv_batched: 16 tile groups x 96 column groups are more than ten cells per
+    CTA, so every CTA rebuilds its activation image in the middle of its range (after eight passes with up
+    to eight vectors, after four with more) and most CTAs cross a tile-group boundary; K leaves a float16
+    tail of 16.  Rows around the tile-group boundaries and random ones, every vector."""
+    from paper_2609_35465_b200 import tetra as tt
+    N, K = 8192, 24 * 384 + 16
+    m = make_matrix(23, 7 + batch, N, K, True, batch=batch)
+    table = tt.tetra_build_table(synth.DEFAULT_GAIN)
+    packed = tt.tetra_pack_codes(torch.from_numpy(m["codes"]).cuda(), table, N, m["B"])
+    y = torch.full((batch, N), float("nan"), dtype=torch.float32, device="cuda")
+    tt.tetra_gemv_batched(packed, torch.from_numpy(m["sigma"]).cuda(), table, torch.from_numpy(m["x"]).cuda(), y, N, K,
+                          batch, torch.from_numpy(m["tail"]).cuda())
+    torch.cuda.synchronize()
+    yh = y.cpu().numpy()
+    assert np.isfinite(yh).all()
+    edges = [0, 31, 32, 511, 512, 513, 1023, 1024, 4095, 4096, 7679, 7680, 8190, 8191]
+    rows = np.unique(np.concatenate([edges, np.random.default_rng(batch).integers(0, N, 18)]))
+    for b in range(batch):
+        ref = oracle_product(orc, m, synth.DEFAULT_GAIN, rows=rows, batch_index=b, threads=4)
+        assert_gemv_close(yh[b][rows], ref, "long ranges, batch %d vector %d" % (batch, b))
