@@ -14,7 +14,11 @@
  *     legacy default stream) and the call does not synchronise, except where
  *     stated;
  *   - arguments are validated on the host before anything is launched; a
- *     rejected call launches nothing.
+ *     rejected call launches nothing;
+ *   - the entry points may be called from several host threads at once (the
+ *     library's one-time set-up per device is guarded); calls that share a
+ *     workspace, an output buffer or tetra_gemv_noalloc's scratch array are
+ *     ordered by the caller (same stream, or events).
  *
  * Word, file order ("canonical"): six little-endian bytes; fields from the
  * least significant bit: i1[11] i2[11] i3[11] s8[6] b1[1] b2[4] b3[1] p[1] r[1]
