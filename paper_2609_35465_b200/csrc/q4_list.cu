@@ -402,7 +402,7 @@ int tetra_q4_list_run(void* workspace_dev, int G, void* stream) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     unsigned char* ws = static_cast<unsigned char*>(workspace_dev);
     cudaError_t e = launch_pdl(k_q4_list_prepare, sms * 2, 256, 0, s, ws);
-    if (e == cudaSuccess) e = G == 128 ? run_main<128, 3>(ws, sms, s) : run_main<64, 6>(ws, sms, s);
+    if (e == cudaSuccess) e = G == 128 ? run_main<128, 2>(ws, sms, s) : run_main<64, 6>(ws, sms, s);
     if (e == cudaSuccess) e = launch_pdl(k_q4_list_combine, sms * 4, 256, 0, s, ws);
     return e == cudaSuccess ? TETRA_OK : TETRA_ERR_CUDA;
 }

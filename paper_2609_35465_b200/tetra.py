@@ -101,6 +101,38 @@ def _ptr(t):
     return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(0)
 
 
+def _need(t, nbytes: int, what: str, cuda: bool = True):
+    """The tensor handed over as `what` holds at least nbytes, contiguously, where the call reads or writes it.
+    The C ABI sees plain pointers; a tensor that is too small would be read or written past its end."""
+    if t is None:
+        return
+    have = t.numel() * t.element_size()
+    if have < nbytes:
+        raise TetraError("%s: tensor of %d bytes, the call needs %d" % (what, have, nbytes))
+    if not t.is_contiguous():
+        raise TetraError("%s: tensor is not contiguous" % what)
+    if cuda and not (t.is_cuda or t.is_pinned()):  # pinned host memory is mapped into the device's address space
+        raise TetraError("%s: tensor is neither on the device nor in pinned host memory" % what)
+
+
+def _blocks(K: int, tail_rule: bool) -> int:
+    return K // BLOCK if (tail_rule or K % BLOCK == 0) else -(-K // BLOCK)
+
+
+def _need_gemv(what, codes, row_scales, x, y, N, K, batch, tail, tail_rule):
+    """Sizes of the tensors of one product (tail_rule: floor(K/24) words per row plus a float16 tail)."""
+    if N <= 0 or K <= 0 or batch <= 0:
+        return  # the library rejects the shape
+    B = _blocks(K, tail_rule)
+    if B > 0:
+        _need(codes, -(-N // 8) * B * 48, what + " codes")
+    _need(row_scales, 4 * N, what + " row_scales")
+    _need(x, 2 * batch * K, what + " x")
+    _need(y, 4 * batch * N, what + " y")
+    if tail_rule and K % BLOCK:
+        _need(tail, 2 * N * (K % BLOCK), what + " tail")
+
+
 # ---------------------------------------------------------------------------
 def tetra_table_bytes() -> int:
     return lib().tetra_table_bytes()
@@ -161,6 +193,7 @@ def tetra_decode_packed(packed: torch.Tensor, table: torch.Tensor, N: int, nbloc
 
 def tetra_gemv(codes, row_scales, table, x, y, N: int, K: int, batch: int = 1, stream=None):
     """Zero-pad rule: ceil(K/24) words per row."""
+    _need_gemv("tetra_gemv", codes, row_scales, x, y, N, K, batch, None, False)
     _check(lib().tetra_gemv(_ptr(codes), _ptr(row_scales), _ptr(table), _ptr(x), _ptr(y), N, K, batch,
                             _stream(stream)), "tetra_gemv")
     return y
@@ -168,6 +201,7 @@ def tetra_gemv(codes, row_scales, table, x, y, N: int, K: int, batch: int = 1, s
 
 def tetra_gemv_tail(codes, row_scales, table, x, y, N: int, K: int, batch: int = 1, tail=None, stream=None):
     """The paper's rule: floor(K/24) words per row plus a float16 tail."""
+    _need_gemv("tetra_gemv_tail", codes, row_scales, x, y, N, K, batch, tail, tail is not None)
     _check(lib().tetra_gemv_tail(_ptr(codes), _ptr(row_scales), _ptr(table), _ptr(x), _ptr(y), N, K, batch,
                                  _ptr(tail), _stream(stream)), "tetra_gemv_tail")
     return y
@@ -178,6 +212,8 @@ def make_problems(items):
     items = list(items)
     arr = (Problem * len(items))()
     for i, it in enumerate(items):
+        _need_gemv("problem %d" % i, it["codes"], it["row_scales"], it["x"], it["y"], it["N"], it["K"], 1, it.get("tail"),
+                   it.get("tail") is not None)
         arr[i] = Problem(it["codes"].data_ptr(), it["row_scales"].data_ptr(), it["x"].data_ptr(),
                          it["tail"].data_ptr() if it.get("tail") is not None else None,
                          it["y"].data_ptr(), it["N"], it["K"])
@@ -242,6 +278,7 @@ def tetra_gemv_noalloc(codes, row_scales, table, x, y, N: int, K: int, tail=None
     """Batch-1 product for callers that may not allocate device memory: the
     scratch buffer lives inside the library (a fixed array, K <= NOALLOC_MAX_K).
     Calls on one device share that array, so they must not overlap on the GPU."""
+    _need_gemv("tetra_gemv_noalloc", codes, row_scales, x, y, N, K, 1, tail, tail is not None)
     _check(lib().tetra_gemv_noalloc(_ptr(codes), _ptr(row_scales), _ptr(table), _ptr(x), _ptr(y), N, K,
                                     _ptr(tail), _stream(stream)), "tetra_gemv_noalloc")
     return y
@@ -254,6 +291,7 @@ def tetra_batched_workspace_bytes(N: int, K: int) -> int:
 def tetra_gemv_batched(codes, row_scales, table, x, y, N: int, K: int, batch: int, tail=None, workspace=None,
                        stream=None):
     """1..16 activation vectors at once: decode once per block, tensor-core contraction per block."""
+    _need_gemv("tetra_gemv_batched", codes, row_scales, x, y, N, K, batch, tail, tail is not None)
     if workspace is None:
         workspace = torch.empty(tetra_batched_workspace_bytes(N, K), dtype=torch.uint8, device=y.device)
     _check(lib().tetra_gemv_batched(_ptr(codes), _ptr(row_scales), _ptr(table), _ptr(x), _ptr(y), N, K, batch,
@@ -275,17 +313,33 @@ def tetra_q4_packed_bytes(N: int, K: int, G: int) -> int:
 def tetra_q4_pack(q, scale, offset, N: int, K: int, G: int, stream=None):
     """File-order matrix (uint8 [N, K/2], float16 [N, K/G] x 2, all on the device) -> packed device buffer."""
     packed = torch.empty(tetra_q4_packed_bytes(N, K, G), dtype=torch.uint8, device=q.device)
+    _need(q, N * (K // 2), "tetra_q4_pack q")
+    _need(scale, 2 * N * (K // G), "tetra_q4_pack scale")
+    _need(offset, 2 * N * (K // G), "tetra_q4_pack offset")
     _check(lib().tetra_q4_pack(_ptr(q), _ptr(scale), _ptr(offset), _ptr(packed), packed.numel(), N, K, G,
                                _stream(stream)), "tetra_q4_pack")
     return packed
 
 
+def _need_q4(what, packed, x, y, N, K, G, batch):
+    n = lib().tetra_q4_packed_bytes(N, K, G)
+    if n == 0 or batch <= 0:
+        return  # the library rejects the shape
+    _need(packed, n, what + " packed")
+    _need(x, 2 * batch * K, what + " x")
+    _need(y, 4 * batch * N, what + " y")
+
+
 def tetra_q4_gemv(packed, x, y, N: int, K: int, G: int, batch: int = 1, stream=None):
+    _need_q4("tetra_q4_gemv", packed, x, y, N, K, G, batch)
     _check(lib().tetra_q4_gemv(_ptr(packed), _ptr(x), _ptr(y), N, K, G, batch, _stream(stream)), "tetra_q4_gemv")
     return y
 
 
 def tetra_q4_rows(packed, ids, out, N: int, K: int, G: int, stream=None):
+    _need_q4("tetra_q4_rows", packed, None, None, N, K, G, 1)
+    _need(ids, 4 * int(ids.numel()), "tetra_q4_rows ids")
+    _need(out, 2 * int(ids.numel()) * K, "tetra_q4_rows out")
     _check(lib().tetra_q4_rows(_ptr(packed), _ptr(ids), int(ids.numel()), _ptr(out), N, K, G, _stream(stream)),
            "tetra_q4_rows")
     return out
@@ -294,6 +348,8 @@ def tetra_q4_rows(packed, ids, out, N: int, K: int, G: int, stream=None):
 def tetra_encode_blocks(w, table, sigma=None, want_cosine=True, stream=None):
     """w: float32 [n, 24] on the device -> (codes uint8 [n, 6] in file order, cosines float32 [n] or None)."""
     n = w.numel() // 24
+    _need(w, 4 * 24 * n, "tetra_encode_blocks w")
+    _need(sigma, 4 * n, "tetra_encode_blocks sigma")
     codes = torch.empty((n, 6), dtype=torch.uint8, device=w.device)
     cos = torch.empty(n, dtype=torch.float32, device=w.device) if want_cosine else None
     _check(lib().tetra_encode_blocks(_ptr(w), _ptr(sigma), _ptr(table), _ptr(codes), _ptr(cos), n, _stream(stream)),

@@ -213,3 +213,36 @@ def test_q4_list_rejects_bad_lists():
     assert tetra.lib().tetra_q4_list_workspace_bytes(bad, 1, 128) == 0        # K not a multiple of G
     ws = torch.empty(16, dtype=torch.uint8, device="cuda")
     assert tetra.lib().tetra_q4_list_plan(ok, 1, 128, ws.data_ptr(), 16, None) == -6
+
+
+def test_binding_rejects_tensors_that_are_too_small():
+    """The C ABI takes plain pointers; the Python binding knows the tensors' sizes and refuses a call whose
+    tensors are smaller than what the call would read or write, before anything is launched."""
+    import torch
+    from paper_2609_35465_b200 import tetra
+    N, K, G = 64, 256, 64
+    q = torch.zeros((N // 2, K // 2), dtype=torch.uint8, device="cuda")          # half the rows
+    sc = torch.ones((N, K // G), dtype=torch.float16, device="cuda")
+    with pytest.raises(tetra.TetraError, match="needs"):
+        tetra.tetra_q4_pack(q, sc, sc, N, K, G)
+    q = torch.zeros((N, K // 2), dtype=torch.uint8, device="cuda")
+    packed = tetra.tetra_q4_pack(q, sc, sc, N, K, G)
+    x = torch.zeros(K, dtype=torch.float16, device="cuda")
+    y = torch.zeros(N, dtype=torch.float32, device="cuda")
+    with pytest.raises(tetra.TetraError, match="needs"):
+        tetra.tetra_q4_gemv(packed[:-16], x, y, N, K, G, 1)
+    with pytest.raises(tetra.TetraError, match="needs"):
+        tetra.tetra_q4_gemv(packed, x, y, N, K, G, 2)                           # two vectors, tensors for one
+    table = tetra.tetra_build_table()
+    codes = torch.zeros(tetra.tetra_codes_bytes(N, 4), dtype=torch.uint8, device="cuda")
+    rs = torch.ones(N, dtype=torch.float32, device="cuda")
+    x = torch.zeros(96, dtype=torch.float16, device="cuda")
+    for call in (lambda: tetra.tetra_gemv(codes, rs, table, x, y, N, 24 * 5),     # five words per row, codes hold four
+                 lambda: tetra.tetra_gemv(codes, rs[:10], table, x, y, N, 96),
+                 lambda: tetra.tetra_gemv_batched(codes, rs, table, x, y, N, 96, 3),
+                 lambda: tetra.tetra_gemv_noalloc(codes, rs, table, x, y[:8], N, 96),
+                 lambda: tetra.make_problems([dict(codes=codes, row_scales=rs, x=x[:50], y=y, N=N, K=96)])):
+        with pytest.raises(tetra.TetraError, match="needs"):
+            call()
+    tetra.tetra_gemv(codes, rs, table, x, y, N, 96)                             # the right sizes pass
+    torch.cuda.synchronize()
