@@ -153,3 +153,52 @@ def test_batched_long_cta_ranges_sampled_rows(orc, batch):
     for b in range(batch):
         ref = oracle_product(orc, m, synth.DEFAULT_GAIN, rows=rows, batch_index=b, threads=4)
         assert_gemv_close(yh[b][rows], ref, "long ranges, batch %d vector %d" % (batch, b))
+
+
+def test_tall_matrix_sampled_rows(orc):
+    """151,936 x 4096 (the row count of the model's vocabulary; 155 MB of codes, 18,992 row groups): the index
+    arithmetic of every path far beyond the projection shapes.  One launch, the planned list, three vectors
+    through the tensor-core kernel; rows at both ends, around the tile-group edges and random ones."""
+    from paper_2609_35465_b200 import tetra as tt
+    N, K, batch = 151936, 4096, 3
+    B, ntail = K // 24, K % 24
+    table = tt.tetra_build_table(synth.DEFAULT_GAIN)
+    codes = synth.codes_torch(31, 4, N, B, device="cuda")
+    packed = tt.tetra_pack_codes(codes, table, N, B)
+    del codes
+    sigma = synth.row_scales(31, 4, N)
+    x = synth.activations(31, 4, K, batch)
+    tail = synth.tails(31, 4, sigma, ntail)
+    d = dict(codes=packed, row_scales=torch.from_numpy(sigma).cuda(), x=torch.from_numpy(x).cuda(),
+             tail=torch.from_numpy(tail).cuda(), N=N, K=K)
+    edges = [0, 7, 8, 511, 512, 75967, 75968, 151424, 151934, 151935]
+    rows = np.unique(np.concatenate([edges, np.random.default_rng(9).integers(0, N, 22)]))
+    host_codes = np.stack([synth.words_to_bytes(synth.words(31, 4, B, int(r) * B)) for r in rows])
+
+    def check(y, b, what):
+        mm = dict(N=len(rows), K=K, B=B, ntail=ntail, codes=host_codes, sigma=sigma[rows], x=x, tail=tail[rows])
+        ref = oracle_product(orc, mm, synth.DEFAULT_GAIN, batch_index=b, threads=4)
+        assert_gemv_close(y[rows], ref, what)
+
+    y = torch.full((batch, N), float("nan"), dtype=torch.float32, device="cuda")
+    d["y"] = y
+    tt.tetra_gemv_tail(packed, d["row_scales"], table, d["x"], y, N, K, 1, d["tail"])
+    torch.cuda.synchronize()
+    y0 = y[0].cpu().numpy()
+    assert np.isfinite(y0).all()
+    check(y0, 0, "tall matrix, one launch")
+    y.fill_(float("nan"))
+    pr = tt.make_problems([d])
+    ws = torch.empty(tt.tetra_grouped_workspace_bytes(pr), dtype=torch.uint8, device="cuda")
+    tt.tetra_gemv_grouped(pr, table, ws)
+    torch.cuda.synchronize()
+    y1 = y[0].cpu().numpy()
+    assert np.isfinite(y1).all()
+    check(y1, 0, "tall matrix, planned list")
+    y.fill_(float("nan"))
+    tt.tetra_gemv_batched(packed, d["row_scales"], table, d["x"], y, N, K, batch, d["tail"])
+    torch.cuda.synchronize()
+    yb = y.cpu().numpy()
+    assert np.isfinite(yb).all()
+    for b in range(batch):
+        check(yb[b], b, "tall matrix, batched vector %d" % b)
