@@ -130,8 +130,17 @@ struct PlanHeader {
     uint32_t off_counters;  // int32 per row group: slices of the group that have finished
     uint32_t off_partials;  // float [row group][slice][8]
     int32_t total_groups;
-    int32_t pad_[3];
+    // coarse mode with unit ranges: units [0, dyn_start) are cut into the warps' ranges; the units from
+    // dyn_start on are claimed one at a time through dyn_next by warps that have finished their range
+    // (k_prepare_x sets dyn_next = dyn_start before every run)
+    int32_t dyn_start;
+    int32_t dyn_next;
+    int32_t pad_[1];
 };
+#ifndef TETRA_DYN_PERMILLE
+#define TETRA_DYN_PERMILLE 100
+#endif
+constexpr int kDynamicTailPermille = TETRA_DYN_PERMILLE;  // share of the list's work left for the claimed units
 
 struct FineInfo {
     int32_t slices;          // column slices per row group
@@ -223,6 +232,8 @@ __global__ void __launch_bounds__(256) k_prepare_x(unsigned char* __restrict__ w
 #pragma unroll
         for (int k = 0; k < 5; ++k) xq[size_t(gc) * 5 + k] = make_uint4(q[4 * k], q[4 * k + 1], q[4 * k + 2], q[4 * k + 3]);
     }
+    if (!H->off_fine && blockIdx.x == 0 && threadIdx.x == 0)
+        reinterpret_cast<PlanHeader*>(ws)->dyn_next = H->dyn_start;  // the claimed units start over
     if (H->off_fine) {  // fine mode: the per-row-group arrival counters start every run at zero
         int32_t* counters = reinterpret_cast<int32_t*>(ws + H->off_counters);
         for (int g = blockIdx.x * blockDim.x + threadIdx.x; g < H->total_groups; g += gridDim.x * blockDim.x)
@@ -248,7 +259,7 @@ constexpr int kUnitThreads = TETRA_UNIT_THREADS;
 constexpr int kUnitWarps = kUnitThreads / 32;
 
 // Coarse mode: every warp walks its range of units (up to three row groups of one matrix, all columns).
-__device__ __forceinline__ void units_coarse(const unsigned char* __restrict__ ws, unsigned char* smem, uint32_t sm_tab) {
+__device__ __forceinline__ void units_coarse(unsigned char* __restrict__ ws, unsigned char* smem, uint32_t sm_tab) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float* red = reinterpret_cast<float*>(smem + kFastBytes) + warp * kRedFloats;
     const PlanHeader* H = reinterpret_cast<const PlanHeader*>(ws);
@@ -263,11 +274,13 @@ __device__ __forceinline__ void units_coarse(const unsigned char* __restrict__ w
     // (warps in grid)-th unit.
     const int gw = blockIdx.x * kUnitWarps + warp, nw = gridDim.x * kUnitWarps;
     int u = gw, u_end = total_units, u_step = nw;
+    bool claim = false;  // after the range: claim the units from dyn_start on, one at a time
     if (H->nwarps == nw) {
         const int32_t* warp_start = reinterpret_cast<const int32_t*>(ws + H->off_warp_start);
         u = __ldg(warp_start + gw);
         u_end = __ldg(warp_start + gw + 1);
         u_step = 1;
+        claim = H->dyn_start < total_units;
     }
     int p = -1, p_begin = 0, p_end = 0;  // matrix of the current unit and its range of units
     // per matrix, kept in registers across its units (everything else is re-read where it is needed)
@@ -282,7 +295,21 @@ __device__ __forceinline__ void units_coarse(const unsigned char* __restrict__ w
     const uint32_t ring = sm_tab + uint32_t(kFastBytes) + uint32_t(kUnitWarps * kRedFloats * 4) + uint32_t(warp) * 3072u + uint32_t(lane) * 16u;
     int pass_parity = 0;
 
-    for (; u < u_end; u += u_step) {
+    for (;; u += u_step) {
+        if (u >= u_end) {
+            if (!claim) break;
+            // The range is done: claim one of the units that were left unassigned.  One atomic per unit; it
+            // only hands out numbers, nothing waits on it, and the numbers a warp gets increase, so the walk
+            // below still only goes up.  (Claiming one unit ahead would hide the atomic's latency but keeps a
+            // register live across the passes, which costs more than it saves.)
+            int c = 0;
+            if (lane == 0) c = atomicAdd(&reinterpret_cast<PlanHeader*>(ws)->dyn_next, 1);
+            c = __shfl_sync(0xFFFFFFFFu, c, 0);
+            if (c >= total_units) break;
+            u = c;
+            u_end = c + 1;
+            have_record = false;
+        }
         if (u >= p_end) {  // first unit, or the walk has left the matrix: units only go up
             do { ++p; p_end = __ldg(unit_prefix + p + 1); } while (u >= p_end);
             p_begin = __ldg(unit_prefix + p);
@@ -605,6 +632,24 @@ cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, 
         };
         long long total = 0;
         for (int i = 0; i < count; ++i) total += unit_work(i) * problem_units(problems_host[i]);
+        // The last tenth of the work is not assigned: warps that finish early claim it unit by unit, which
+        // evens out what the cost model and the SMs' unequal speeds leave (measured on the Qwen3-8B pass:
+        // the average scheduler idled 4.2 % of the kernel's time behind the slowest one).  Only when a warp
+        // has at least a few units.
+        H->dyn_start = int32_t(units);
+        if (units >= 8LL * nwarps) {
+            const long long planned = total - total * kDynamicTailPermille / 1000;
+            long long acc = 0;
+            int i = 0;
+            while (i < count - 1 && acc + unit_work(i) * problem_units(problems_host[i]) <= planned) {
+                acc += unit_work(i) * problem_units(problems_host[i]);
+                ++i;
+            }
+            long long ds = up[i] + (planned - acc) / unit_work(i);
+            if (ds > units) ds = units;
+            H->dyn_start = int32_t(ds);
+            total = acc + (ds - up[i]) * unit_work(i);
+        }
         int32_t* wsx = reinterpret_cast<int32_t*>(buf + H->off_warp_start);
         int pi = 0;
         long long before = 0;  // work of matrices 0..pi-1
@@ -615,10 +660,10 @@ cudaError_t grouped_plan(const Problem* problems_host, int count, void* ws_dev, 
                 ++pi;
             }
             long long uu = up[pi] + (target - before) / unit_work(pi);
-            if (uu > units) uu = units;
+            if (uu > H->dyn_start) uu = H->dyn_start;
             wsx[w] = int32_t(uu);
         }
-        wsx[nwarps] = int32_t(units);
+        wsx[nwarps] = H->dyn_start;
     }
     // pageable source: the runtime stages it before returning, so the buffer can be freed
     if (e == cudaSuccess) e = cudaMemcpyAsync(ws_dev, buf, meta, cudaMemcpyHostToDevice, s);
