@@ -29,6 +29,7 @@ namespace {
 
 constexpr int kQ4ListThreads = 512;
 constexpr int kQ4ListWarps = kQ4ListThreads / 32;
+constexpr int kPieceFloats = 32;  // a partial strip: column 0 of its 32 rows (the list call has one vector per matrix)
 
 struct Q4Item {
     const unsigned char* packed;
@@ -59,7 +60,7 @@ Q4ListLayout list_layout(int count, size_t total_groups, int nwarps) {
     L.off_items = align256(sizeof(Q4ListHeader));
     L.off_gs = align256(L.off_items + size_t(count) * sizeof(Q4Item));
     L.off_pieces = align256(L.off_gs + total_groups * 64);
-    L.off_piece_strip = align256(L.off_pieces + size_t(nwarps) * 2 * 1024);
+    L.off_piece_strip = align256(L.off_pieces + size_t(nwarps) * 2 * kPieceFloats * 4);
     L.total = align256(L.off_piece_strip + size_t(nwarps) * 2 * 4);
     return L;
 }
@@ -83,9 +84,14 @@ __global__ void __launch_bounds__(256) k_q4_list_prepare(unsigned char* __restri
     float2* gs = reinterpret_cast<float2*>(ws + H->off_gs);
     int32_t* piece_strip = reinterpret_cast<int32_t*>(ws + H->off_piece_strip);
     const int G = H->G, sub = threadIdx.x & 7;
+    // the matrices' first groups go to shared memory: the search below would otherwise be a chain of
+    // dependent loads from L2 that is most of this kernel's time
+    __shared__ uint32_t group_begin_sm[TETRA_Q4_LIST_MAX];
+    for (int i = threadIdx.x; i < H->count; i += blockDim.x) group_begin_sm[i] = items[i].group_begin;
+    __syncthreads();
     for (uint32_t gg = (blockIdx.x * blockDim.x + threadIdx.x) >> 3; gg < H->total_groups;
          gg += (gridDim.x * blockDim.x) >> 3) {
-        const int it = find_item(H->count, gg, [&](int i) { return items[i].group_begin; });
+        const int it = find_item(H->count, gg, [&](int i) { return group_begin_sm[i]; });
         const uint2* src = reinterpret_cast<const uint2*>(items[it].x + size_t(gg - items[it].group_begin) * G);
         float lo = 0.f, hi = 0.f;  // k % 4 in {0, 1} / {2, 3}
         for (int i = 0; i < G / 32; ++i) {
@@ -244,10 +250,11 @@ __global__ void __launch_bounds__(kQ4ListThreads, 1) k_q4_list_main(unsigned cha
                             if (row < I.N) I.y[row] = acc[h][i];
                         }
                 }
-            } else {  // a strip shared with a neighbouring warp: leave a piece
-                float* mine = pieces + size_t(2 * gw + n_pieces) * 256 + 8 * lane;
-                *reinterpret_cast<float4*>(mine) = make_float4(acc[0][0], acc[0][1], acc[0][2], acc[0][3]);
-                *reinterpret_cast<float4*>(mine + 4) = make_float4(acc[1][0], acc[1][1], acc[1][2], acc[1][3]);
+            } else {  // a strip shared with a neighbouring warp: leave a piece (column 0: row 16 h + g + 8 j at 4 g' ...)
+                if (t == 0) {  // floats 4 g .. 4 g + 3 = rows g, g + 8, 16 + g, 24 + g
+                    float* mine = pieces + size_t(2 * gw + n_pieces) * kPieceFloats + 4 * g;
+                    *reinterpret_cast<float4*>(mine) = make_float4(acc[0][0], acc[0][2], acc[1][0], acc[1][2]);
+                }
                 if (lane == 0) piece_strip[2 * gw + n_pieces] = int32_t(I.strip_begin) + strip;
                 ++n_pieces;
             }
@@ -262,36 +269,37 @@ __global__ void __launch_bounds__(kQ4ListThreads, 1) k_q4_list_main(unsigned cha
     q4_cp_async_wait<0>();
 }
 
-// Block i looks at piece i (pieces are in memory order: warp, then first/second): if it is the first
-// piece of its strip, the block adds the strip's pieces in that order and stores column 0.
+// Warp i looks at piece slot i (slots are in memory order: warp, then first/second): if it holds the first
+// piece of its strip, the warp adds the strip's pieces in slot order and stores the 32 rows.
 __global__ void __launch_bounds__(256) k_q4_list_combine(unsigned char* __restrict__ ws) {
     pdl_release();
+    const int lane = threadIdx.x & 31;
+    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     pdl_wait();
     const Q4ListHeader* H = reinterpret_cast<const Q4ListHeader*>(ws);
-    const Q4Item* items = reinterpret_cast<const Q4Item*>(ws + H->off_items);
-    const float* pieces = reinterpret_cast<const float*>(ws + H->off_pieces);
-    const int32_t* piece_strip = reinterpret_cast<const int32_t*>(ws + H->off_piece_strip);
     const int npieces = 2 * H->nwarps;
-    for (int i = blockIdx.x; i < npieces; i += gridDim.x) {
-        const int sid = piece_strip[i];
-        if (sid < 0) continue;
-        int j = i - 1;
-        while (j >= 0 && piece_strip[j] < 0) --j;
-        if (j >= 0 && piece_strip[j] == sid) continue;  // not the first piece of its strip
-        const int e = threadIdx.x, lane = e >> 3, h = (e >> 2) & 1, ii = e & 3;
-        float total = 0.f;
-        for (int k = i; k < npieces; ++k) {
-            const int s = piece_strip[k];
-            if (s < 0) continue;
-            if (s != sid) break;
-            total += pieces[size_t(k) * 256 + e];
-        }
-        const int col = 2 * (lane & 3) + (ii & 1);
-        if (col != 0) continue;
-        const int it = find_item(H->count, uint32_t(sid), [&](int q) { return items[q].strip_begin; });
-        const int row = 32 * (sid - int(items[it].strip_begin)) + 16 * h + (lane >> 2) + 8 * (ii >> 1);
-        if (row < items[it].N) items[it].y[row] = total;
+    if (i >= npieces) return;
+    const int32_t* piece_strip = reinterpret_cast<const int32_t*>(ws + H->off_piece_strip);
+    const int sid = piece_strip[i];
+    if (sid < 0) return;
+    // a strip has at most one piece per warp: its earlier pieces, if any, sit in the slots just before
+    int j = i - 1;
+    while (j >= 0 && piece_strip[j] < 0) --j;
+    if (j >= 0 && piece_strip[j] == sid) return;  // not the first piece of its strip
+    const float* pieces = reinterpret_cast<const float*>(ws + H->off_pieces);
+    float total = 0.f;
+    for (int k = i; k < npieces; ++k) {
+        const int s = piece_strip[k];
+        if (s < 0) continue;
+        if (s != sid) break;
+        total += pieces[size_t(k) * kPieceFloats + lane];
     }
+    const Q4Item* items = reinterpret_cast<const Q4Item*>(ws + H->off_items);
+    const int it = find_item(H->count, uint32_t(sid), [&](int q) { return items[q].strip_begin; });
+    // float 4 g + j of a piece is row g + 8 (j & 1) + 16 (j >> 1) of the strip
+    const int g = lane >> 2, jj = lane & 3;
+    const int row = 32 * (sid - int(items[it].strip_begin)) + g + 8 * (jj & 1) + 16 * (jj >> 1);
+    if (row < items[it].N) items[it].y[row] = total;
 }
 
 int check_list(const tetra_q4_problem* p, int count, int G) {
@@ -403,7 +411,7 @@ int tetra_q4_list_run(void* workspace_dev, int G, void* stream) {
     unsigned char* ws = static_cast<unsigned char*>(workspace_dev);
     cudaError_t e = launch_pdl(k_q4_list_prepare, sms * 2, 256, 0, s, ws);
     if (e == cudaSuccess) e = G == 128 ? run_main<128, 2>(ws, sms, s) : run_main<64, 6>(ws, sms, s);
-    if (e == cudaSuccess) e = launch_pdl(k_q4_list_combine, sms * 4, 256, 0, s, ws);
+    if (e == cudaSuccess) e = launch_pdl(k_q4_list_combine, (2 * sms * kQ4ListWarps + 7) / 8, 256, 0, s, ws);  // a warp per piece slot
     return e == cudaSuccess ? TETRA_OK : TETRA_ERR_CUDA;
 }
 
