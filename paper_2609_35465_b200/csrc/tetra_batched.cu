@@ -354,9 +354,16 @@ k_combine_batched(const float* __restrict__ partials, const float* __restrict__ 
     pdl_wait();  // the pieces come from k_gemv_batched
     if (!mine) return;
     const float* p = partials + (size_t(first + tg) * kBatWarps + warp) * kPieceFloats + rt * (8 * NG) + v;
+    // sixteen pieces are loaded at a time (all of them, for the usual split of a tile group over about twenty
+    // CTAs, in two rounds of independent loads) and added in piece order
     float total = 0.f;
-#pragma unroll 8
-    for (uint32_t k = 0; k < pieces; ++k) total += __ldcg(p + size_t(k) * kBatWarps * kPieceFloats);
+    for (uint32_t k0 = 0; k0 < pieces; k0 += 16) {
+        float v[16];
+#pragma unroll
+        for (uint32_t j = 0; j < 16; ++j) v[j] = k0 + j < pieces ? __ldcg(p + size_t(k0 + j) * kBatWarps * kPieceFloats) : 0.f;
+#pragma unroll
+        for (uint32_t j = 0; j < 16; ++j) total += v[j];
+    }
     float res = scale * total;
     const int ntail = tail ? K % 24 : 0;
     for (int k = 0; k < ntail; ++k)
