@@ -193,9 +193,11 @@ int tetra_gemv_grouped(const tetra_problem *problems_host, int count, const void
  * least tetra_batched_workspace_bytes(N, K) bytes (partial results of column
  * ranges, which a second small kernel sums in a fixed order; its contents need
  * no initialisation), private to the call until it completes.  Two kernel
- * launches; the result is bit-identical from run to run.  With one or two
- * vectors the call runs tetra_gemv_tail's kernel instead (one launch, the
- * workspace untouched), which is faster there. */
+ * launches; the result is bit-identical from run to run.  With one vector
+ * the call runs tetra_gemv_tail's kernel instead (one launch, the workspace
+ * untouched), which is faster there; two to four vectors run a kernel that
+ * feeds the tensor cores from the decoder's registers, five and more one
+ * that goes through shared-memory tiles. */
 size_t tetra_batched_workspace_bytes(int N, int K);
 int tetra_gemv_batched(const void *codes, const float *row_scales, const void *table,
                        const void *x, float *y, int N, int K, int batch, const void *tail,

@@ -12,7 +12,7 @@ using namespace tetra;
 namespace {
 
 constexpr int kMaxBlocksPerRow = 2048;  // K <= 49,152
-constexpr int kBatchedMinVectors = 3;   // tetra_gemv_batched runs the tensor-core kernel from this many vectors on
+constexpr int kBatchedMinVectors = 2;   // tetra_gemv_batched runs the tensor-core kernel from this many vectors on
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
@@ -231,8 +231,8 @@ int tetra_gemv_batched(const void* codes, const float* row_scales, const void* t
     const int B = tail_mode ? K / 24 : (K + 23) / 24;
     if (B <= 0 || B > kMaxBlocksPerRow) return TETRA_ERR_SHAPE;
     if (workspace_bytes < batched_workspace_bytes(N, B)) return TETRA_ERR_SIZE;
-    // One or two vectors: decoding once per vector in the single-launch kernel is faster than the
-    // tensor-core path's fixed costs (measured on B200: 11.5 / 21 us against 24 us on 4096 x 12288).
+    // One vector: the single-launch kernel is faster than the tensor-core paths' fixed costs (measured on
+    // B200, 4096 x 12288: 11.6 us against 15.8 us for two vectors on the tensor cores).
     if (batch <= kBatchedMinVectors - 1)
         return tetra_gemv_tail(codes, row_scales, table, x, y, N, K, batch, tail, stream);
     return cuda_status(launch_gemv_batched(codes, row_scales, table, x, y, N, K, batch, (K % 24) ? tail : nullptr,

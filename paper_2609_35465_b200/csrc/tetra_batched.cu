@@ -1,4 +1,5 @@
-// Decode-and-multiply for 2..16 activation vectors at once (Eq. (2), Sec. 5.1).
+// Decode-and-multiply for 2..16 activation vectors at once (Eq. (2), Sec. 5.1): k_gemv_batched (5..16
+// vectors, described first) and k_gemv_few (2..4 vectors, further down).
 //
 // A block is decoded once and multiplied with every vector, so the decode cost
 // is shared.  The products over a block's 24 coordinates for up to 16 vectors
@@ -25,8 +26,7 @@
 // row scale and the tail.  The only waits are CTA barriers, cp.async groups and griddepcontrol.wait.
 #include <cuda_fp16.h>
 
-#include "tetra_device.cuh"
-#include "tetra_launch.h"
+#include "tetra_gemv_common.cuh"
 
 namespace tetra {
 
@@ -332,6 +332,233 @@ k_gemv_batched(const DeviceTables* __restrict__ tab, const unsigned char* __rest
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Two to four vectors: the same cells, rings, image chunks and pieces as k_gemv_batched, but no shared-memory
+// tile between decoder and tensor cores.  Lane 4 q + t decodes, for each of the warp's two row blocks, rows
+// 2 q and 2 q + 1 at column t of the pass's four columns; the MMA takes eight coordinates of both blocks
+// from every lane as A (rows q and q + 8), and B is block diagonal -- column 2 t + plane of B is zero outside
+// the k range that lane t feeds -- so D[q][2 t + plane] is the dot product of lane (q, t)'s own block with
+// its own column's activation plane and arrives in that same lane.  Three MMAs (coordinate pairs) times two
+// B sets (unsigned middle and low planes; signed high plane) per vector and row block.  The activation
+// image holds, per (column quad, vector), the B fragments as they are read: three 128-byte lines (one per
+// coordinate pair: bytes 0..63 middle and low planes, entry 2 t + plane; 64..95 high plane, entry t;
+// 96..103 zero, read by the lanes whose part of B is zero), the four columns' steps at 104 + 4 t of line 0.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kQuadBytes = 384;
+constexpr int kFewMaxVectors = 4;
+constexpr int kFewChunkPasses = 16;  // passes whose image is held at a time: 16 x 4 vectors x 384 bytes = 24 KiB
+
+__device__ __forceinline__ void mma_bd(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                       uint32_t b1, const int (&c)[4], bool b_signed) {
+    if (b_signed)
+        asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+            : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(c[0]), "r"(c[1]), "r"(c[2]), "r"(c[3]));
+    else
+        asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+            : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(c[0]), "r"(c[1]), "r"(c[2]), "r"(c[3]));
+}
+
+template <int V>
+__global__ void __launch_bounds__(kBatThreads, 1)
+k_gemv_few(const DeviceTables* __restrict__ tab, const unsigned char* __restrict__ codes, const __half* __restrict__ x,
+           int N, int K, int B, float* __restrict__ partials, int tile_groups, int col_groups) {
+    constexpr int RB = 2, PC = 4, CP = kFewChunkPasses;
+    constexpr int kPieceFloats = RB * 128;  // the piece layout of k_gemv_batched<1, 2>: 32 rows x 8 vector slots
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    pdl_release();
+    unsigned char* smem = stage_fast_tables_async(tab, smem_raw);
+    const uint32_t sm_tab = smem_u32(smem);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int q = lane >> 2, t = lane & 3;
+    const uint32_t ring = smem_u32(smem + kFastBytes) + uint32_t(warp) * (2 * kBatRingSlot);
+    const uint32_t image = smem_u32(smem + kFastBytes) + uint32_t(kBatWarps) * (2 * kBatRingSlot);
+    unsigned char* image_ptr = smem + kFastBytes + kBatWarps * (2 * kBatRingSlot);
+    const int row_groups = (N + 7) / 8;
+    const uint32_t Bu = uint32_t(B);
+    // the lane's words in a slot: rows 2 q, 2 q + 1 of row block rb sit in row group 2 rb + q / 4, part (q / 2) % 2
+    const uint32_t lane_w0 = uint32_t(q >> 2) * kBatRingGroup + uint32_t((q >> 1) & 1) * 64u + uint32_t(t) * 16u + uint32_t(q & 1) * 8u;
+    const uint32_t lane_w1 = uint32_t(q >> 2) * kBatRingGroup + 128u + uint32_t(t) * 16u + uint32_t(q & 3) * 4u;
+    // this lane's part of the B fragments (the other lanes read the zeros)
+    const uint32_t lane_x1 = (q >> 1) == t ? uint32_t(q) * 8u : 96u;
+    const uint32_t lane_x2 = q == 2 * t ? 64u + uint32_t(t) * 8u : 96u;
+    const uint32_t lane_xs = 104u + 4u * uint32_t(t);
+    const uint32_t cp0_gp = uint32_t(lane >> 2), cp1_gp = 8u + uint32_t(lane >> 2), cp_col = uint32_t(lane & 3);
+    const uint32_t cp0_dst = (cp0_gp / 3u) * kBatRingGroup + (cp0_gp % 3u) * 64u + cp_col * 16u;
+    const uint32_t cp1_dst = (cp1_gp / 3u) * kBatRingGroup + (cp1_gp % 3u) * 64u + cp_col * 16u;
+
+    const uint32_t ctas = gridDim.x, cells = uint32_t(tile_groups) * uint32_t(col_groups), CG = uint32_t(col_groups);
+    const uint32_t cell_begin = uint32_t(uint64_t(blockIdx.x) * cells / ctas);
+    const uint32_t cell_end = uint32_t((uint64_t(blockIdx.x) + 1) * cells / ctas);
+    uint32_t tg = cell_begin / CG, cg = cell_begin - tg * CG;
+
+    auto fetch = [&](uint32_t ftg, uint32_t fcg, uint32_t slot) {
+        const uint32_t G0 = (ftg * kBatWarps + uint32_t(warp)) * (2 * RB);
+        const uint32_t col = fcg * PC + cp_col;
+        const bool in = col < Bu;
+        const uint4* base = reinterpret_cast<const uint4*>(codes) + size_t(G0) * 3 * Bu + (in ? col : 0u);
+        const uint32_t dst = ring + slot * kBatRingSlot;
+        const bool have0 = in && G0 + cp0_gp / 3u < uint32_t(row_groups);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(dst + cp0_dst),
+                     "l"(have0 ? base + size_t(cp0_gp) * Bu : reinterpret_cast<const uint4*>(codes)), "r"(have0 ? 16u : 0u));
+        if (lane < 16) {
+            const bool have1 = in && G0 + cp1_gp / 3u < uint32_t(row_groups);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(dst + cp1_dst),
+                         "l"(have1 ? base + size_t(cp1_gp) * Bu : reinterpret_cast<const uint4*>(codes)), "r"(have1 ? 16u : 0u));
+        }
+        asm volatile("cp.async.commit_group;");
+    };
+    if (cell_begin < cell_end) fetch(tg, cg, 0);
+    else asm volatile("cp.async.commit_group;");
+    pdl_wait();  // x may come from the preceding kernel; the partial results of an earlier call have been read
+
+    // Image of a chunk of CP passes: thread (pass i, column cs, vector v) quantises one column of one vector and
+    // writes its planes into the quad's record as B fragments.
+    auto image_build = [&](uint32_t first_cell) {
+        for (int id = threadIdx.x; id < CP * PC * V; id += kBatThreads) {
+            const int v = id % V, cs = (id / V) % PC, i = id / (V * PC);
+            const uint32_t cell = first_cell + uint32_t(i);
+            if (cell >= cell_end) continue;
+            const int col = int(cell % CG) * PC + cs;
+            uint32_t qv[20];
+            if (col < B) {
+                quantise_column(x + size_t(v) * K, K, col, qv);
+            } else {
+#pragma unroll
+                for (int k = 0; k < 20; ++k) qv[k] = 0u;
+            }
+            unsigned char* rec = image_ptr + size_t(i * V + v) * kQuadBytes;
+#pragma unroll
+            for (int pr = 0; pr < 3; ++pr) {
+                unsigned char* line = rec + 128 * pr;
+                *reinterpret_cast<uint2*>(line + 16 * cs) = make_uint2(qv[6 + 2 * pr], qv[7 + 2 * pr]);        // middle plane
+                *reinterpret_cast<uint2*>(line + 16 * cs + 8) = make_uint2(qv[12 + 2 * pr], qv[13 + 2 * pr]);  // low plane
+                *reinterpret_cast<uint2*>(line + 64 + 8 * cs) = make_uint2(qv[2 * pr], qv[2 * pr + 1]);        // high plane
+                if (cs == 0) *reinterpret_cast<uint2*>(line + 96) = make_uint2(0u, 0u);
+            }
+            *reinterpret_cast<uint32_t*>(rec + 104 + 4 * cs) = qv[18];
+        }
+    };
+    image_build(cell_begin);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();  // tables staged, first image built
+
+    float acc[RB][2][V];
+#pragma unroll
+    for (int rb = 0; rb < RB; ++rb)
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int v = 0; v < V; ++v) acc[rb][j][v] = 0.f;
+
+    for (uint32_t cell = cell_begin; cell < cell_end; ++cell) {
+        const uint32_t pass = cell - cell_begin, slot = pass & 1u, in_chunk = pass % CP;
+        const bool active = (int(tg) * kBatWarps + warp) * (16 * RB) < N;  // warp-uniform
+        uint32_t ntg = tg, ncg = cg + 1;
+        if (ncg == CG) { ncg = 0; ++ntg; }
+        if (in_chunk == 0 && pass > 0) {  // CTA-uniform: the image of the next chunk of passes replaces the old one
+            __syncthreads();
+            image_build(cell);
+            __syncthreads();
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncwarp();  // every lane's copies have landed, and every lane has left the other slot
+        if (cell + 1 < cell_end) fetch(ntg, ncg, slot ^ 1u);
+        if (active) {
+            const uint32_t src = ring + slot * kBatRingSlot;
+            FastBlock f[RB][2];
+            float scale[RB][2];
+#pragma unroll
+            for (int rb = 0; rb < RB; ++rb) {
+                uint2 w0;
+                uint32_t w1pair;
+                asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(w0.x), "=r"(w0.y) : "r"(src + lane_w0 + rb * 2 * kBatRingGroup));
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w1pair) : "r"(src + lane_w1 + rb * 2 * kBatRingGroup));
+                fast_decode<false>(sm_tab, w0.x, w1pair, f[rb][0]);
+                fast_decode<true>(sm_tab, w0.y, w1pair, f[rb][1]);
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    int n2 = int(f[rb][j].goff);
+#pragma unroll
+                    for (int k = 0; k < 6; ++k) n2 = dp4a_ss(f[rb][j].y[k], f[rb][j].y[k], n2);
+                    scale[rb][j] = lds32f(uint32_t(n2));
+                }
+            }
+            const uint32_t img = image + in_chunk * (V * kQuadBytes);
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                uint2 bm[3], bh[3];
+#pragma unroll
+                for (int pr = 0; pr < 3; ++pr) {
+                    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(bm[pr].x), "=r"(bm[pr].y) : "r"(img + v * kQuadBytes + 128 * pr + lane_x1));
+                    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(bh[pr].x), "=r"(bh[pr].y) : "r"(img + v * kQuadBytes + 128 * pr + lane_x2));
+                }
+                float step;
+                asm volatile("ld.shared.f32 %0, [%1];" : "=f"(step) : "r"(img + v * kQuadBytes + lane_xs));
+                if constexpr (V <= 2) {  // registers allow the two row blocks' MMA chains side by side
+                int dm[RB][4], dh[RB][4];
+#pragma unroll
+                for (int rb = 0; rb < RB; ++rb)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) { dm[rb][i] = 0; dh[rb][i] = 0; }
+#pragma unroll
+                for (int pr = 0; pr < 3; ++pr)
+#pragma unroll
+                    for (int rb = 0; rb < RB; ++rb) {
+                        mma_bd(dm[rb], f[rb][0].y[2 * pr], f[rb][1].y[2 * pr], f[rb][0].y[2 * pr + 1], f[rb][1].y[2 * pr + 1],
+                               bm[pr].x, bm[pr].y, dm[rb], false);
+                        mma_bd(dh[rb], f[rb][0].y[2 * pr], f[rb][1].y[2 * pr], f[rb][0].y[2 * pr + 1], f[rb][1].y[2 * pr + 1],
+                               bh[pr].x, bh[pr].y, dh[rb], true);
+                    }
+#pragma unroll
+                for (int rb = 0; rb < RB; ++rb) {
+                    const int dot0 = dh[rb][0] * 65536 + (dm[rb][0] * 256 + dm[rb][1]);
+                    const int dot1 = dh[rb][2] * 65536 + (dm[rb][2] * 256 + dm[rb][3]);
+                    acc[rb][0][v] = fmaf(float(dot0), scale[rb][0] * step, acc[rb][0][v]);
+                    acc[rb][1][v] = fmaf(float(dot1), scale[rb][1] * step, acc[rb][1][v]);
+                }
+                } else {
+#pragma unroll
+                for (int rb = 0; rb < RB; ++rb) {
+                    int dm[4] = {0, 0, 0, 0}, dh[4] = {0, 0, 0, 0};
+#pragma unroll
+                    for (int pr = 0; pr < 3; ++pr) {
+                        mma_bd(dm, f[rb][0].y[2 * pr], f[rb][1].y[2 * pr], f[rb][0].y[2 * pr + 1], f[rb][1].y[2 * pr + 1],
+                               bm[pr].x, bm[pr].y, dm, false);
+                        mma_bd(dh, f[rb][0].y[2 * pr], f[rb][1].y[2 * pr], f[rb][0].y[2 * pr + 1], f[rb][1].y[2 * pr + 1],
+                               bh[pr].x, bh[pr].y, dh, true);
+                    }
+                    // exact int32 dot products of -y with the 24-bit activations (the scale carries the other minus sign)
+                    const int dot0 = dh[0] * 65536 + (dm[0] * 256 + dm[1]);
+                    const int dot1 = dh[2] * 65536 + (dm[2] * 256 + dm[3]);
+                    acc[rb][0][v] = fmaf(float(dot0), scale[rb][0] * step, acc[rb][0][v]);
+                    acc[rb][1][v] = fmaf(float(dot1), scale[rb][1] * step, acc[rb][1][v]);
+                }
+                }
+            }
+        }
+        if (cell + 1 == cell_end || ntg != tg) {  // CTA-uniform: this CTA's piece of tile group tg is complete
+            // the four lanes of a row (its four columns) are added, then lane t = 0 writes the row's V sums
+            float* mine = partials + (size_t(blockIdx.x + tg) * kBatWarps + warp) * kPieceFloats;
+#pragma unroll
+            for (int rb = 0; rb < RB; ++rb)
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+#pragma unroll
+                    for (int v = 0; v < V; ++v) {
+                        float sum = acc[rb][j][v];
+                        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
+                        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
+                        if (t == 0) mine[(16 * rb + 2 * q + j) * 8 + v] = sum;
+                        acc[rb][j][v] = 0.f;
+                    }
+        }
+        tg = ntg;
+        cg = ncg;
+    }
+}
+
 // Sum of a tile group's pieces in CTA order, row scale, tail (Sec. 5.1): one thread per (row, vector).
 template <int NG, int RB>
 __global__ void __launch_bounds__(256)
@@ -427,6 +654,21 @@ static cudaError_t launch_variant(const void* codes, const float* row_scales, co
                               y, N, K, B, batch, P.tile_groups, P.col_groups, P.ctas);
 }
 
+template <int V>
+static cudaError_t launch_few(const void* codes, const float* row_scales, const void* table, const __half* xh, float* y,
+                              int N, int K, int B, const __half* tl, float* partials, int sms, cudaStream_t s) {
+    const uint32_t smem = kTableSmemBytes + kBatWarps * 2 * kBatRingSlot + kFewChunkPasses * kFewMaxVectors * kQuadBytes;
+    static PerDeviceOnce once;
+    cudaError_t e = once.run([smem] { return cudaFuncSetAttribute(k_gemv_few<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)); });
+    if (e != cudaSuccess) return e;
+    const BatchedPlan P = batched_plan(N, B, 2, sms);
+    e = launch_pdl(k_gemv_few<V>, P.ctas, kBatThreads, smem, s, static_cast<const DeviceTables*>(table),
+                   static_cast<const unsigned char*>(codes), xh, N, K, B, partials, P.tile_groups, P.col_groups);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(k_combine_batched<1, 2>, int((size_t(N) * 8 + 255) / 256), 256, 0, s, static_cast<const float*>(partials),
+                      row_scales, xh, tl, y, N, K, B, V, P.tile_groups, P.col_groups, P.ctas);
+}
+
 cudaError_t launch_gemv_batched(const void* codes, const float* row_scales, const void* table, const void* x,
                                 float* y, int N, int K, int batch, const void* tail, void* ws, cudaStream_t s) {
     int sms = 0;
@@ -446,6 +688,11 @@ cudaError_t launch_gemv_batched(const void* codes, const float* row_scales, cons
     const __half* xh = static_cast<const __half*>(x);
     const __half* tl = static_cast<const __half*>(tail);
     float* partials = static_cast<float*>(ws);
+#ifndef TETRA_NO_FEW
+    if (batch == 2) return launch_few<2>(codes, row_scales, table, xh, y, N, K, B, tl, partials, sms, s);
+    if (batch == 3) return launch_few<3>(codes, row_scales, table, xh, y, N, K, B, tl, partials, sms, s);
+    if (batch == 4) return launch_few<4>(codes, row_scales, table, xh, y, N, K, B, tl, partials, sms, s);
+#endif
     if (batch <= 8)
         return launch_variant<1, TETRA_BAT_RB1>(codes, row_scales, table, xh, y, N, K, B, batch, tl, partials, sms, smem, s);
     return launch_variant<2, TETRA_BAT_RB2>(codes, row_scales, table, xh, y, N, K, B, batch, tl, partials, sms, smem, s);
