@@ -27,7 +27,6 @@ namespace tetra {
 static_assert(kListMax == TETRA_LIST_MAX, "list length limit must agree with the header");
 
 constexpr int kChunkGroups = 32;  // row groups whose partial sums share the shared-memory buffer
-constexpr int kTailStage = 23;    // float16 tail values per row staged in shared memory (K mod 24 <= 23)
 
 struct ListSmem {
     // offsets from the 16 KiB-aligned table copy; total includes the alignment slack
