@@ -131,14 +131,16 @@ def test_down_proj_batched_sampled_rows(orc, batch):
         assert_gemv_close(yh[b][rows], ref, "batched, batch %d vector %d" % (batch, b))
 
 
-@pytest.mark.parametrize("batch", [5, 16])
-def test_batched_long_cta_ranges_sampled_rows(orc, batch):
+@pytest.mark.parametrize("batch,words", [(5, 384), (16, 384), (2, 640), (4, 640)])
+def test_batched_long_cta_ranges_sampled_rows(orc, batch, words):
     """8192 x 9232 through tetra_gemv_batched: 16 tile groups x 96 column groups are more than ten cells per
-    CTA, so every CTA rebuilds its activation image in the middle of its range (after eight passes with up
+    CTA, so every CTA rebuilds its activation image in the middle of its range (after eight passes with five
     to eight vectors, after four with more) and most CTAs cross a tile-group boundary; K leaves a float16
-    tail of 16.  Rows around the tile-group boundaries and random ones, every vector."""
+    tail of 16.  With two to four vectors (another kernel, whose image holds sixteen passes) 8192 x 15376:
+    160 column groups, seventeen cells per CTA.  Rows around the tile-group boundaries and random ones, every
+    vector."""
     from paper_2609_35465_b200 import tetra as tt
-    N, K = 8192, 24 * 384 + 16
+    N, K = 8192, 24 * words + 16
     m = make_matrix(23, 7 + batch, N, K, True, batch=batch)
     table = tt.tetra_build_table(synth.DEFAULT_GAIN)
     packed = tt.tetra_pack_codes(torch.from_numpy(m["codes"]).cuda(), table, N, m["B"])
