@@ -111,7 +111,10 @@ int tetra_decode_packed(const void *packed_dev, const void *table_dev, int8_t *y
  * codes: packed layout of an N x ceil(K/24) matrix (16-byte aligned).
  * row_scales: float32 [N].  x: float16 [batch][K] (2-byte aligned; 16-byte
  * aligned rows are faster).  y: float32 [batch][N], fully overwritten.
- * 1 <= batch <= 16.
+ * 1 <= batch <= 16.  The call takes no scratch memory, so with batch > 1 the
+ * vectors are multiplied one after another inside one launch (every word is
+ * decoded once per vector); tetra_gemv_batched decodes once for all vectors
+ * and is the faster call from two vectors on.
  * Arithmetic: the 24 activations of a block column are held as 24-bit fixed
  * point with a power-of-two step 2^(E-22), 2^E <= max |x_j| < 2^(E+1) over the
  * column; the products with the lattice coordinates and their sum over the
